@@ -1,0 +1,188 @@
+/*
+ * eco.h -- C-ABI of the B200 (sm_100a) ECO optimizer-step library.
+ *
+ * ECO (arXiv 2601.22101) trains with quantized weights and NO master weights:
+ * each step dequantizes the stored weight, applies the optimizer update,
+ * requantizes, and injects the quantization error into the momentum buffer
+ * (Algorithm 1 = OPTIM_STEP followed by ECO_QUANTIZE; Algorithm 2 for momentum
+ * SGD, Algorithm 3 for Adam; quantizer and rounding of Sec. 3.1).
+ *
+ * All pointers named "device" are CUDA device pointers of the device the
+ * context was created on; the caller owns every buffer and the stream.  The
+ * library owns only its descriptor tables and a few bytes of reduction
+ * scratch per tensor.  No call in this header synchronizes the device unless
+ * it says so.  There is no CPU fallback: without a CUDA device every call
+ * that needs one returns ECO_ERR_CUDA.
+ */
+#ifndef ECO_H_
+#define ECO_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct eco_ctx eco_ctx;
+
+typedef enum eco_status {
+    ECO_OK = 0,
+    ECO_ERR_INVALID_ARG = 1, /* a value outside the domain of the method (see eco_step) */
+    ECO_ERR_UNSUPPORTED = 2, /* a combination this build has no kernel for */
+    ECO_ERR_ALIGNMENT = 3,   /* a buffer is not 16-byte aligned */
+    ECO_ERR_CUDA = 4,        /* a CUDA runtime call failed; eco_last_error has its text */
+    ECO_ERR_NOMEM = 5,
+    ECO_ERR_TIMEOUT = 6      /* reserved for bounded device-side waits */
+} eco_status;
+
+/* Weight format (Sec. 3.1; rho = largest representable magnitude). */
+enum { ECO_FORMAT_FP8_E4M3 = 0, /* OCP E4M3 "FN": bias 7, rho = 448, S.1111.111 = NaN is never written;
+                                   one byte per element */
+       ECO_FORMAT_INT4 = 1 };   /* integers -7..7, rho = 7, two's-complement nibbles, two per byte,
+                                   element 2k in the low nibble; -8 is never written */
+/* Scale granularity (Sec. 3.1, "granularity").  Tensors are row-major [rows, cols]. */
+enum { ECO_SCALE_PER_TENSOR = 0, /* 1 scale                                              */
+       ECO_SCALE_PER_ROW = 1,    /* rows scales                                          */
+       ECO_SCALE_PER_BLOCK = 2 };/* rows * ceil(cols / block) scales, blocks of `block`
+                                    consecutive elements of one row; the last block of a
+                                    row may be short                                     */
+enum { ECO_SCALE_F32 = 0, ECO_SCALE_BF16 = 1 };
+enum { ECO_OPT_SGDM = 0,  /* dampened momentum SGD: m~ = beta m + (1-beta) g, theta~ = theta^ - eta m~ (Eq. 2-3) */
+       ECO_OPT_ADAM = 1 };/* Adam in the form of Sec. 3.2, "Adam"                                                */
+enum { ECO_ROUND_NEAREST = 0,    /* ties to the even code                                                        */
+       ECO_ROUND_STOCHASTIC = 1 };/* upper neighbour with probability (x - lower)/gap; Philox4x32-10 keyed by
+                                     seed, counter = (element index / 4, tensor_id, step), word = index mod 4;
+                                     the top 24 bits of the word are compared with the fraction                  */
+enum { ECO_INJECT_NONE = 0, /* naive master-weight removal (Sec. 3.4): the error is dropped */
+       ECO_INJECT_ECO = 1 };/* the paper's method: m^ = m~ + alpha e                        */
+
+typedef struct eco_config {
+    int32_t format;      /* ECO_FORMAT_*                                  */
+    int32_t granularity; /* ECO_SCALE_PER_*                               */
+    int32_t block;       /* block length for ECO_SCALE_PER_BLOCK: 128     */
+    int32_t scale_dtype; /* ECO_SCALE_F32 or ECO_SCALE_BF16               */
+    int32_t optimizer;   /* ECO_OPT_*                                     */
+    int32_t rounding;    /* ECO_ROUND_*                                   */
+    int32_t injection;   /* ECO_INJECT_*; ECO_INJECT_ECO is the method    */
+    int32_t reserved;    /* must be 0                                     */
+} eco_config;
+
+/* One parameter tensor and its optimizer state.  All buffers are device
+ * memory, 16-byte aligned, contiguous, and must not overlap one another. */
+typedef struct eco_tensor {
+    void* w;           /* in/out: codes; rows*cols bytes (FP8) or rows*cols/2 bytes (INT4)        */
+    void* scale;       /* in/out: scales, layout given by granularity, dtype by scale_dtype       */
+    const void* grad;  /* in: gradient, bf16 [rows*cols]; re-read at every eco_step                */
+    float* m;          /* in/out: first moment / momentum, f32 [rows*cols]                         */
+    float* v;          /* in/out: second moment, f32 [rows*cols]; must be NULL for ECO_OPT_SGDM    */
+    int64_t rows, cols;
+    uint32_t tensor_id;/* selects the tensor's random stream; unique within a context              */
+    uint32_t reserved; /* must be 0                                                                */
+} eco_tensor;
+
+/*
+ * eco_create -- bind a list of tensors that share one configuration.
+ * Operation: prepares Algorithm 1 for the tensor list (host-side only apart
+ * from one upload of the descriptor table).
+ *   out      host; receives the context.
+ *   cfg      host; copied.
+ *   tensors  host array of n entries; copied (the device buffers they name are
+ *            NOT copied and must outlive the context).
+ *   device   CUDA device ordinal; made current for the calling thread.
+ * Errors: ECO_ERR_INVALID_ARG (NULL, n == 0, rows/cols < 1, rows*cols >= 2^34,
+ * INT4 with odd cols, duplicate tensor_id, v not matching the optimizer,
+ * overlapping buffers, non-device pointers), ECO_ERR_UNSUPPORTED (block != 128,
+ * unknown enum), ECO_ERR_ALIGNMENT, ECO_ERR_CUDA, ECO_ERR_NOMEM.  On error *out
+ * is NULL and eco_last_error(NULL) describes the failure.  Allocates device
+ * memory (tables and scratch); synchronizes the device once.
+ */
+eco_status eco_create(eco_ctx** out, const eco_config* cfg, const eco_tensor* tensors, size_t n, int device);
+
+/*
+ * eco_step -- one quantized training step t on every tensor of the context
+ * (Algorithm 1): for each element
+ *   theta^ = value(code) * scale                         (Sec. 3.1)
+ *   SGDM:  m~ = beta1 m + (1-beta1) g ; theta~ = theta^ - lr m~          (Eq. 2-3)
+ *   Adam:  m~, v~ updated with g ; theta~ = theta^ - lr (m~/(1-beta1^t)) / (sqrt(v~/(1-beta2^t)) + eps)
+ *   scale' = max|theta~| / rho over the element's scale block ; code' = round(theta~ / scale')
+ *   e = theta~ - value(code') * scale'                   (Algorithm 2/3, line 2)
+ *   SGDM:  m = m~ + (1/lr)(1 - 1/beta1) e                (Algorithm 2, line 5)
+ *   Adam:  m = m~ + ((1-beta1^t)/lr)(1 - 1/beta1)(sqrt(v~/(1-beta2^t)) + eps) e ; v = v~   (Algorithm 3, line 5)
+ * and writes code', scale', m, v in place.  No full-precision weight is ever stored.
+ *   step   t >= 1, the 1-based count of updates including this one.
+ *   seed   key of the stochastic-rounding stream (ignored for ECO_ROUND_NEAREST).
+ *   beta2, eps are ignored for ECO_OPT_SGDM.
+ *   cuda_stream  a cudaStream_t (NULL = the legacy default stream).
+ * Asynchronous: enqueues its kernels on cuda_stream and returns; it never
+ * synchronizes and never allocates.  Consecutive steps of one context must be
+ * ordered on the device (same stream, or events), because they share the
+ * context's reduction scratch.
+ * Errors: ECO_ERR_INVALID_ARG for lr <= 0 or non-finite (alpha = (1/lr)(..) is
+ * undefined, Eq. 7), beta1 outside (0,1) (1/beta1), Adam beta2 outside (0,1),
+ * eps < 0, step < 1; ECO_ERR_CUDA for a failed launch.  On ECO_ERR_INVALID_ARG
+ * nothing is launched and no buffer is modified.
+ */
+eco_status eco_step(eco_ctx* ctx, float lr, float beta1, float beta2, float eps,
+                    uint64_t step, uint64_t seed, void* cuda_stream);
+
+/*
+ * eco_step_host -- the same step for callers that keep the state in HOST
+ * memory (offloaded optimizer state).  `tensors` has the layout of eco_tensor
+ * but every pointer is a host pointer (pinned memory makes the copies
+ * asynchronous and faster).  Per tensor group the call copies codes, scales,
+ * gradient and moments to device staging buffers it allocates, runs the
+ * kernels of eco_step, copies codes, scales and moments back, and returns
+ * after synchronizing its internal streams.  h2d_bytes / d2h_bytes (host,
+ * optional) receive the bytes copied in each direction.
+ * Errors: as eco_create and eco_step; ECO_ERR_NOMEM if staging cannot be allocated.
+ */
+eco_status eco_step_host(const eco_config* cfg, const eco_tensor* tensors, size_t n, int device,
+                         float lr, float beta1, float beta2, float eps, uint64_t step, uint64_t seed,
+                         uint64_t* h2d_bytes, uint64_t* d2h_bytes);
+
+/* eco_destroy -- free the context's tables and scratch (synchronizes the device). NULL is allowed. */
+eco_status eco_destroy(eco_ctx* ctx);
+
+/* eco_last_error -- text of the last failure of `ctx`, or of the calling thread's last failed
+ * call when ctx is NULL.  The pointer stays valid until the next call on that context / thread. */
+const char* eco_last_error(const eco_ctx* ctx);
+
+/*
+ * eco_quantize -- theta^_0 = q(theta_0): the symmetric quantizer of Sec. 3.1
+ * (scale = max|x| / rho per scale block, zero-point 0) used to initialise the
+ * quantized state (Appendix A, initialisation).
+ *   x      device, in: f32 [rows*cols], 16-byte aligned.
+ *   w, scale  device, out: layouts as in eco_tensor.
+ *   cfg->optimizer and cfg->injection are ignored; rounding, seed, step and
+ *   tensor_id select the rounding exactly as in eco_step (use step 0 for the
+ *   initial state).
+ * Asynchronous on cuda_stream except for one temporary device allocation when
+ * granularity is ECO_SCALE_PER_TENSOR (freed stream-ordered).
+ * Errors: as eco_create.
+ */
+eco_status eco_quantize(const eco_config* cfg, const float* x, int64_t rows, int64_t cols,
+                        void* w, void* scale, uint64_t seed, uint64_t step, uint32_t tensor_id,
+                        int device, void* cuda_stream);
+
+/*
+ * eco_set_option -- process-wide tuning knobs read by the NEXT eco_create:
+ *   "l2_group_bytes"  per-tensor scales only: bytes of inputs one pass-1/pass-2 launch pair
+ *                     covers, so that pass 2 re-reads from L2 (-1 = half the L2 size, the
+ *                     default; 0 = one pair for the whole context)
+ *   "reverse_pass2"   per-tensor scales only: 1 (default) walks pass 2 in the opposite order
+ *                     of pass 1 so that it starts with the most recently read data
+ * No option changes any result bit.  Errors: ECO_ERR_INVALID_ARG for an unknown name.
+ */
+eco_status eco_set_option(const char* name, int64_t value);
+
+/* eco_num_launches -- number of kernels one eco_step of this context enqueues. */
+int eco_num_launches(const eco_ctx* ctx);
+
+/* eco_version -- "major.minor.patch" of the library. */
+const char* eco_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ECO_H_ */

@@ -1,0 +1,538 @@
+// C-ABI of the ECO step library: argument validation, the work-unit tables,
+// per-step scalar derivation and kernel enqueueing.  Declarations and the
+// full contract of every entry point are in include/eco.h.
+#include <algorithm>
+#include <cmath>
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <string>
+#include <unordered_set>
+#include <vector>
+
+#include "../../include/eco.h"
+#include "eco_launch.h"
+
+using eco::LaunchConfig;
+using eco::StepParams;
+using eco::TensorDesc;
+
+namespace {
+
+thread_local std::string g_thread_error;
+
+enum LaunchKind { KIND_BLOCK_FAST = 0, KIND_BLOCK_GENERIC = 1, KIND_TENSOR = 2, KIND_ROW = 3 };
+
+struct Launch {
+    int kind;
+    size_t desc_offset;   // into d_descs
+    size_t unit_offset;   // into d_unit_tensor
+    uint32_t n_units;
+};
+
+// Options settable through eco_set_option before eco_create.
+struct Options {
+    int64_t l2_group_bytes = -1;   // per-tensor scale: input bytes per launch pair; -1 = half of the L2 size, 0 = one group
+    int64_t reverse_pass2 = 1;     // per-tensor scale: walk pass 2 in the opposite order of pass 1
+};
+Options g_options;
+
+}  // namespace
+
+struct eco_ctx {
+    eco_config cfg;
+    int device = 0;
+    LaunchConfig lc{};
+    std::vector<Launch> launches;
+    TensorDesc* d_descs = nullptr;
+    uint32_t* d_unit_tensor = nullptr;
+    uint32_t* d_amax[2] = {nullptr, nullptr};
+    float* d_s_old = nullptr;
+    uint64_t calls = 0;
+    bool reverse_pass2 = true;
+    int num_launches = 0;
+    std::string err;
+};
+
+namespace {
+
+eco_status fail(eco_ctx* ctx, eco_status st, const char* fmt, ...) {
+    char buf[512];
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(buf, sizeof buf, fmt, ap);
+    va_end(ap);
+    g_thread_error = buf;
+    if (ctx) ctx->err = buf;
+    return st;
+}
+
+#define ECO_CUDA(ctx, call)                                                                        \
+    do {                                                                                           \
+        cudaError_t e_ = (call);                                                                   \
+        if (e_ != cudaSuccess)                                                                     \
+            return fail(ctx, e_ == cudaErrorMemoryAllocation ? ECO_ERR_NOMEM : ECO_ERR_CUDA,       \
+                        "%s failed: %s", #call, cudaGetErrorString(e_));                           \
+    } while (0)
+
+eco_status check_config(const eco_config* cfg, bool need_optimizer) {
+    if (!cfg) return fail(nullptr, ECO_ERR_INVALID_ARG, "cfg is NULL");
+    if (cfg->format != ECO_FORMAT_FP8_E4M3 && cfg->format != ECO_FORMAT_INT4)
+        return fail(nullptr, ECO_ERR_UNSUPPORTED, "unknown format %d", cfg->format);
+    if (cfg->granularity < ECO_SCALE_PER_TENSOR || cfg->granularity > ECO_SCALE_PER_BLOCK)
+        return fail(nullptr, ECO_ERR_UNSUPPORTED, "unknown granularity %d", cfg->granularity);
+    if (cfg->granularity == ECO_SCALE_PER_BLOCK && cfg->block != 128)
+        return fail(nullptr, ECO_ERR_UNSUPPORTED, "block %d: only 128 is built", cfg->block);
+    if (cfg->scale_dtype != ECO_SCALE_F32 && cfg->scale_dtype != ECO_SCALE_BF16)
+        return fail(nullptr, ECO_ERR_UNSUPPORTED, "unknown scale_dtype %d", cfg->scale_dtype);
+    if (cfg->rounding != ECO_ROUND_NEAREST && cfg->rounding != ECO_ROUND_STOCHASTIC)
+        return fail(nullptr, ECO_ERR_UNSUPPORTED, "unknown rounding %d", cfg->rounding);
+    if (need_optimizer) {
+        if (cfg->optimizer != ECO_OPT_SGDM && cfg->optimizer != ECO_OPT_ADAM)
+            return fail(nullptr, ECO_ERR_UNSUPPORTED, "unknown optimizer %d", cfg->optimizer);
+        if (cfg->injection != ECO_INJECT_NONE && cfg->injection != ECO_INJECT_ECO)
+            return fail(nullptr, ECO_ERR_UNSUPPORTED, "unknown injection %d", cfg->injection);
+    }
+    if (cfg->reserved != 0) return fail(nullptr, ECO_ERR_INVALID_ARG, "cfg->reserved must be 0");
+    return ECO_OK;
+}
+
+LaunchConfig launch_config(const eco_config& cfg) {
+    LaunchConfig lc;
+    lc.format = cfg.format == ECO_FORMAT_FP8_E4M3 ? eco::FMT_FP8 : eco::FMT_INT4;
+    lc.optimizer = cfg.optimizer == ECO_OPT_ADAM ? eco::OPT_ADAM : eco::OPT_SGDM;
+    lc.rounding = cfg.rounding == ECO_ROUND_STOCHASTIC ? eco::RND_SR : eco::RND_RTN;
+    lc.bf16_scale = cfg.scale_dtype == ECO_SCALE_BF16 ? 1 : 0;
+    return lc;
+}
+
+uint64_t n_scales(const eco_config& cfg, int64_t rows, int64_t cols) {
+    if (cfg.granularity == ECO_SCALE_PER_TENSOR) return 1;
+    if (cfg.granularity == ECO_SCALE_PER_ROW) return static_cast<uint64_t>(rows);
+    return static_cast<uint64_t>(rows) * static_cast<uint64_t>((cols + cfg.block - 1) / cfg.block);
+}
+
+uint64_t code_bytes(const eco_config& cfg, uint64_t numel) {
+    return cfg.format == ECO_FORMAT_FP8_E4M3 ? numel : (numel + 1) / 2;
+}
+
+uint64_t scale_bytes(const eco_config& cfg, int64_t rows, int64_t cols) {
+    return n_scales(cfg, rows, cols) * (cfg.scale_dtype == ECO_SCALE_BF16 ? 2 : 4);
+}
+
+eco_status check_shape(const eco_config& cfg, int64_t rows, int64_t cols, size_t i) {
+    if (rows < 1 || cols < 1) return fail(nullptr, ECO_ERR_INVALID_ARG, "tensor %zu: rows and cols must be >= 1", i);
+    if (rows >= (int64_t(1) << 34) || cols >= (int64_t(1) << 32) ||
+        static_cast<unsigned __int128>(rows) * static_cast<unsigned __int128>(cols) >= (static_cast<unsigned __int128>(1) << 34))
+        return fail(nullptr, ECO_ERR_INVALID_ARG, "tensor %zu: rows*cols must be < 2^34 and cols < 2^32", i);
+    if (cfg.format == ECO_FORMAT_INT4 && (cols & 1))
+        return fail(nullptr, ECO_ERR_INVALID_ARG, "tensor %zu: INT4 needs an even number of columns", i);
+    return ECO_OK;
+}
+
+eco_status check_device_ptr(const void* p, int device, const char* what, size_t i, bool on_device) {
+    if (!p) return fail(nullptr, ECO_ERR_INVALID_ARG, "tensor %zu: %s is NULL", i, what);
+    if (reinterpret_cast<uintptr_t>(p) & 15) return fail(nullptr, ECO_ERR_ALIGNMENT, "tensor %zu: %s is not 16-byte aligned", i, what);
+    if (on_device) {
+        cudaPointerAttributes attr;
+        cudaError_t e = cudaPointerGetAttributes(&attr, p);
+        if (e != cudaSuccess) {
+            cudaGetLastError();
+            return fail(nullptr, ECO_ERR_CUDA, "cudaPointerGetAttributes(%s of tensor %zu): %s", what, i, cudaGetErrorString(e));
+        }
+        if (attr.type != cudaMemoryTypeDevice && attr.type != cudaMemoryTypeManaged)
+            return fail(nullptr, ECO_ERR_INVALID_ARG, "tensor %zu: %s is not device memory", i, what);
+        if (attr.type == cudaMemoryTypeDevice && attr.device != device)
+            return fail(nullptr, ECO_ERR_INVALID_ARG, "tensor %zu: %s lives on device %d, context is on %d", i, what, attr.device, device);
+    }
+    return ECO_OK;
+}
+
+eco_status check_hyper(eco_ctx* ctx, const eco_config& cfg, float lr, float beta1, float beta2, float eps, uint64_t step) {
+    if (!(lr > 0.0f) || !std::isfinite(lr)) return fail(ctx, ECO_ERR_INVALID_ARG, "lr must be finite and > 0 (got %g)", lr);
+    if (!(beta1 > 0.0f && beta1 < 1.0f)) return fail(ctx, ECO_ERR_INVALID_ARG, "beta1 must be in (0,1) (got %g)", beta1);
+    if (step < 1) return fail(ctx, ECO_ERR_INVALID_ARG, "step is 1-based");
+    if (cfg.optimizer == ECO_OPT_ADAM) {
+        if (!(beta2 > 0.0f && beta2 < 1.0f)) return fail(ctx, ECO_ERR_INVALID_ARG, "beta2 must be in (0,1) (got %g)", beta2);
+        if (!(eps >= 0.0f) || !std::isfinite(eps)) return fail(ctx, ECO_ERR_INVALID_ARG, "eps must be finite and >= 0 (got %g)", eps);
+    }
+    return ECO_OK;
+}
+
+// Scalars of one step, each derived in binary64 from the binary32 arguments and cast once.
+StepParams derive_params(const eco_config& cfg, float lr_f, float beta1_f, float beta2_f, float eps_f,
+                         uint64_t step, uint64_t seed) {
+    const double lr = lr_f, b1 = beta1_f, b2 = beta2_f;
+    const double t = static_cast<double>(step);
+    StepParams P;
+    std::memset(&P, 0, sizeof P);
+    P.beta1 = beta1_f;
+    P.beta2 = beta2_f;
+    P.eps = eps_f;
+    P.one_minus_beta1 = static_cast<float>(1.0 - b1);
+    P.one_minus_beta2 = static_cast<float>(1.0 - b2);
+    P.neg_lr = -lr_f;
+    P.alpha = static_cast<float>((1.0 / lr) * (1.0 - 1.0 / b1));
+    if (cfg.optimizer == ECO_OPT_ADAM) {
+        const double bc1 = 1.0 - std::pow(b1, t);
+        const double bc2 = 1.0 - std::pow(b2, t);
+        P.inv_bc2 = static_cast<float>(1.0 / bc2);
+        P.lr_over_bc1 = static_cast<float>(lr / bc1);
+        P.adam_coef = static_cast<float>((bc1 / lr) * (1.0 - 1.0 / b1));
+    }
+    P.seed_lo = static_cast<uint32_t>(seed);
+    P.seed_hi = static_cast<uint32_t>(seed >> 32);
+    P.step_lo = static_cast<uint32_t>(step);
+    P.step_hi = static_cast<uint32_t>(step >> 32);
+    P.inject = cfg.injection == ECO_INJECT_ECO ? 1 : 0;
+    return P;
+}
+
+struct Interval {
+    uintptr_t lo, hi;
+    size_t tensor;
+    const char* what;
+};
+
+}  // namespace
+
+extern "C" {
+
+const char* eco_version(void) { return "0.1.0"; }
+
+const char* eco_last_error(const eco_ctx* ctx) { return ctx ? ctx->err.c_str() : g_thread_error.c_str(); }
+
+eco_status eco_set_option(const char* name, int64_t value) {
+    if (!name) return fail(nullptr, ECO_ERR_INVALID_ARG, "option name is NULL");
+    if (!std::strcmp(name, "l2_group_bytes")) { g_options.l2_group_bytes = value; return ECO_OK; }
+    if (!std::strcmp(name, "reverse_pass2")) { g_options.reverse_pass2 = value; return ECO_OK; }
+    return fail(nullptr, ECO_ERR_INVALID_ARG, "unknown option '%s'", name);
+}
+
+int eco_num_launches(const eco_ctx* ctx) { return ctx ? ctx->num_launches : 0; }
+
+eco_status eco_create(eco_ctx** out, const eco_config* cfg, const eco_tensor* tensors, size_t n, int device) {
+    if (!out) return fail(nullptr, ECO_ERR_INVALID_ARG, "out is NULL");
+    *out = nullptr;
+    if (eco_status st = check_config(cfg, true)) return st;
+    if (!tensors || n == 0) return fail(nullptr, ECO_ERR_INVALID_ARG, "empty tensor list");
+    if (n > 0x7FFFFFFFu) return fail(nullptr, ECO_ERR_INVALID_ARG, "too many tensors");
+    ECO_CUDA(nullptr, cudaSetDevice(device));
+    cudaDeviceProp prop;
+    ECO_CUDA(nullptr, cudaGetDeviceProperties(&prop, device));
+    if (prop.major < 10) return fail(nullptr, ECO_ERR_UNSUPPORTED, "device %d is sm_%d%d; this library is built for sm_100a", device, prop.major, prop.minor);
+
+    const bool adam = cfg->optimizer == ECO_OPT_ADAM;
+    std::unordered_set<uint32_t> ids;
+    std::vector<Interval> iv;
+    iv.reserve(n * 5);
+    for (size_t i = 0; i < n; ++i) {
+        const eco_tensor& t = tensors[i];
+        if (eco_status st = check_shape(*cfg, t.rows, t.cols, i)) return st;
+        if (t.reserved != 0) return fail(nullptr, ECO_ERR_INVALID_ARG, "tensor %zu: reserved must be 0", i);
+        if (!ids.insert(t.tensor_id).second) return fail(nullptr, ECO_ERR_INVALID_ARG, "tensor %zu: duplicate tensor_id %u", i, t.tensor_id);
+        if (adam && !t.v) return fail(nullptr, ECO_ERR_INVALID_ARG, "tensor %zu: Adam needs v", i);
+        if (!adam && t.v) return fail(nullptr, ECO_ERR_INVALID_ARG, "tensor %zu: v must be NULL for SGDM", i);
+        const uint64_t numel = static_cast<uint64_t>(t.rows) * static_cast<uint64_t>(t.cols);
+        const struct { const void* p; uint64_t bytes; const char* what; } bufs[5] = {
+            {t.w, code_bytes(*cfg, numel), "w"}, {t.scale, scale_bytes(*cfg, t.rows, t.cols), "scale"},
+            {t.grad, numel * 2, "grad"}, {t.m, numel * 4, "m"}, {t.v, numel * 4, "v"}};
+        for (int b = 0; b < (adam ? 5 : 4); ++b) {
+            if (eco_status st = check_device_ptr(bufs[b].p, device, bufs[b].what, i, true)) return st;
+            const uintptr_t lo = reinterpret_cast<uintptr_t>(bufs[b].p);
+            iv.push_back({lo, lo + bufs[b].bytes, i, bufs[b].what});
+        }
+    }
+    std::sort(iv.begin(), iv.end(), [](const Interval& a, const Interval& b) { return a.lo < b.lo; });
+    for (size_t k = 1; k < iv.size(); ++k)
+        if (iv[k].lo < iv[k - 1].hi)
+            return fail(nullptr, ECO_ERR_INVALID_ARG, "buffers overlap: %s of tensor %zu and %s of tensor %zu",
+                        iv[k - 1].what, iv[k - 1].tensor, iv[k].what, iv[k].tensor);
+
+    eco_ctx* ctx = new (std::nothrow) eco_ctx;
+    if (!ctx) return fail(nullptr, ECO_ERR_NOMEM, "out of host memory");
+    ctx->cfg = *cfg;
+    ctx->device = device;
+    ctx->lc = launch_config(*cfg);
+    ctx->reverse_pass2 = g_options.reverse_pass2 != 0;
+
+    // ---- work-unit tables -------------------------------------------------
+    const uint64_t rpu = static_cast<uint64_t>(eco::rows_per_unit());
+    std::vector<TensorDesc> descs;
+    std::vector<uint32_t> unit_tensor;
+    auto base_desc = [&](size_t i) {
+        const eco_tensor& t = tensors[i];
+        TensorDesc d;
+        std::memset(&d, 0, sizeof d);
+        d.w = static_cast<uint8_t*>(t.w);
+        d.scale = t.scale;
+        d.grad = static_cast<const uint16_t*>(t.grad);
+        d.m = t.m;
+        d.v = t.v;
+        d.numel = static_cast<uint64_t>(t.rows) * static_cast<uint64_t>(t.cols);
+        d.cols = static_cast<uint32_t>(t.cols);
+        d.blocks_per_row = static_cast<uint32_t>((t.cols + 127) / 128);
+        d.tensor_id = t.tensor_id;
+        d.slot = static_cast<uint32_t>(i);
+        return d;
+    };
+    // Appends one launch over the tensors `members`; returns false if the grid would overflow.
+    auto add_launch = [&](int kind, const std::vector<size_t>& members) -> bool {
+        if (members.empty()) return true;
+        Launch L;
+        L.kind = kind;
+        L.desc_offset = descs.size();
+        L.unit_offset = unit_tensor.size();
+        uint64_t units = 0;
+        for (size_t k = 0; k < members.size(); ++k) {
+            TensorDesc d = base_desc(members[k]);
+            uint64_t nu;
+            if (kind == KIND_ROW) {
+                d.n_blocks = static_cast<uint64_t>(tensors[members[k]].rows);
+                nu = d.n_blocks;
+            } else {
+                d.n_blocks = (kind == KIND_TENSOR) ? (d.numel + 127) / 128
+                                                   : static_cast<uint64_t>(tensors[members[k]].rows) * d.blocks_per_row;
+                nu = (d.n_blocks + rpu - 1) / rpu;
+            }
+            if (units + nu > 0x7FFFFFFFull) return false;
+            d.first_unit = static_cast<uint32_t>(units);
+            descs.push_back(d);
+            unit_tensor.insert(unit_tensor.end(), static_cast<size_t>(nu), static_cast<uint32_t>(k));
+            units += nu;
+        }
+        L.n_units = static_cast<uint32_t>(units);
+        ctx->launches.push_back(L);
+        return true;
+    };
+
+    bool ok = true;
+    if (cfg->granularity == ECO_SCALE_PER_BLOCK) {
+        std::vector<size_t> fast, generic;
+        for (size_t i = 0; i < n; ++i) ((tensors[i].cols % 128 == 0) ? fast : generic).push_back(i);
+        ok = add_launch(KIND_BLOCK_FAST, fast) && add_launch(KIND_BLOCK_GENERIC, generic);
+        ctx->num_launches = static_cast<int>(ctx->launches.size());
+    } else if (cfg->granularity == ECO_SCALE_PER_ROW) {
+        std::vector<size_t> all(n);
+        for (size_t i = 0; i < n; ++i) all[i] = i;
+        ok = add_launch(KIND_ROW, all);
+        ctx->num_launches = 1;
+    } else {
+        // Per-tensor scale: pass 1 + pass 2 per group of tensors whose inputs fit the L2 budget, so
+        // that pass 2 finds what pass 1 read still cached.
+        int64_t budget = g_options.l2_group_bytes;
+        if (budget < 0) budget = static_cast<int64_t>(prop.l2CacheSize) / 2;
+        const double in_bytes_per_elem = (cfg->format == ECO_FORMAT_FP8_E4M3 ? 1.0 : 0.5) + 2.0 + (adam ? 8.0 : 4.0);
+        std::vector<size_t> group;
+        double group_bytes = 0;
+        for (size_t i = 0; i < n && ok; ++i) {
+            const double b = in_bytes_per_elem * static_cast<double>(tensors[i].rows) * static_cast<double>(tensors[i].cols);
+            if (!group.empty() && budget > 0 && group_bytes + b > static_cast<double>(budget)) {
+                ok = add_launch(KIND_TENSOR, group);
+                group.clear();
+                group_bytes = 0;
+            }
+            group.push_back(i);
+            group_bytes += b;
+        }
+        if (ok) ok = add_launch(KIND_TENSOR, group);
+        ctx->num_launches = 2 * static_cast<int>(ctx->launches.size());
+    }
+    if (!ok) {
+        delete ctx;
+        return fail(nullptr, ECO_ERR_UNSUPPORTED, "tensor list too large for one launch grid");
+    }
+
+    auto cleanup = [&](eco_status st) {
+        eco_destroy(ctx);
+        return st;
+    };
+#define ECO_CUDA_CTX(call)                                                                                  \
+    do {                                                                                                    \
+        cudaError_t e_ = (call);                                                                            \
+        if (e_ != cudaSuccess)                                                                              \
+            return cleanup(fail(nullptr, e_ == cudaErrorMemoryAllocation ? ECO_ERR_NOMEM : ECO_ERR_CUDA,    \
+                                "%s failed: %s", #call, cudaGetErrorString(e_)));                           \
+    } while (0)
+    ECO_CUDA_CTX(cudaMalloc(&ctx->d_descs, descs.size() * sizeof(TensorDesc)));
+    ECO_CUDA_CTX(cudaMalloc(&ctx->d_unit_tensor, std::max<size_t>(unit_tensor.size(), 1) * sizeof(uint32_t)));
+    ECO_CUDA_CTX(cudaMemcpy(ctx->d_descs, descs.data(), descs.size() * sizeof(TensorDesc), cudaMemcpyHostToDevice));
+    ECO_CUDA_CTX(cudaMemcpy(ctx->d_unit_tensor, unit_tensor.data(), unit_tensor.size() * sizeof(uint32_t), cudaMemcpyHostToDevice));
+    if (cfg->granularity == ECO_SCALE_PER_TENSOR) {
+        for (int p = 0; p < 2; ++p) {
+            ECO_CUDA_CTX(cudaMalloc(&ctx->d_amax[p], n * sizeof(uint32_t)));
+            ECO_CUDA_CTX(cudaMemset(ctx->d_amax[p], 0, n * sizeof(uint32_t)));
+        }
+        ECO_CUDA_CTX(cudaMalloc(&ctx->d_s_old, n * sizeof(float)));
+    }
+    ECO_CUDA_CTX(cudaDeviceSynchronize());
+#undef ECO_CUDA_CTX
+    *out = ctx;
+    return ECO_OK;
+}
+
+eco_status eco_step(eco_ctx* ctx, float lr, float beta1, float beta2, float eps,
+                    uint64_t step, uint64_t seed, void* cuda_stream) {
+    if (!ctx) return fail(nullptr, ECO_ERR_INVALID_ARG, "ctx is NULL");
+    if (eco_status st = check_hyper(ctx, ctx->cfg, lr, beta1, beta2, eps, step)) return st;
+    const StepParams P = derive_params(ctx->cfg, lr, beta1, beta2, eps, step, seed);
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    const int parity = static_cast<int>(ctx->calls & 1);
+    for (const Launch& L : ctx->launches) {
+        const TensorDesc* descs = ctx->d_descs + L.desc_offset;
+        const uint32_t* units = ctx->d_unit_tensor + L.unit_offset;
+        switch (L.kind) {
+            case KIND_BLOCK_FAST:
+            case KIND_BLOCK_GENERIC:
+                ECO_CUDA(ctx, eco::launch_block128(ctx->lc, descs, units, L.n_units, L.kind == KIND_BLOCK_GENERIC, P, stream));
+                break;
+            case KIND_ROW:
+                ECO_CUDA(ctx, eco::launch_row(ctx->lc, descs, units, L.n_units, P, stream));
+                break;
+            case KIND_TENSOR:
+                ECO_CUDA(ctx, eco::launch_tensor_amax(ctx->lc, descs, units, L.n_units, P, ctx->d_amax[parity], ctx->d_s_old, stream));
+                ECO_CUDA(ctx, eco::launch_tensor_apply(ctx->lc, descs, units, L.n_units, P, ctx->d_amax[parity],
+                                                       ctx->d_amax[parity ^ 1], ctx->d_s_old, ctx->reverse_pass2, stream));
+                break;
+        }
+    }
+    ctx->calls++;
+    return ECO_OK;
+}
+
+eco_status eco_destroy(eco_ctx* ctx) {
+    if (!ctx) return ECO_OK;
+    cudaSetDevice(ctx->device);
+    cudaDeviceSynchronize();
+    cudaFree(ctx->d_descs);
+    cudaFree(ctx->d_unit_tensor);
+    cudaFree(ctx->d_amax[0]);
+    cudaFree(ctx->d_amax[1]);
+    cudaFree(ctx->d_s_old);
+    delete ctx;
+    return ECO_OK;
+}
+
+eco_status eco_quantize(const eco_config* cfg, const float* x, int64_t rows, int64_t cols,
+                        void* w, void* scale, uint64_t seed, uint64_t step, uint32_t tensor_id,
+                        int device, void* cuda_stream) {
+    if (eco_status st = check_config(cfg, false)) return st;
+    if (eco_status st = check_shape(*cfg, rows, cols, 0)) return st;
+    ECO_CUDA(nullptr, cudaSetDevice(device));
+    if (eco_status st = check_device_ptr(x, device, "x", 0, true)) return st;
+    if (eco_status st = check_device_ptr(w, device, "w", 0, true)) return st;
+    if (eco_status st = check_device_ptr(scale, device, "scale", 0, true)) return st;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    LaunchConfig lc = launch_config(*cfg);
+    eco_config c2 = *cfg;
+    c2.optimizer = ECO_OPT_SGDM;
+    StepParams P = derive_params(c2, 1.0f, 0.5f, 0.5f, 0.0f, step, seed);
+    const uint64_t numel = static_cast<uint64_t>(rows) * static_cast<uint64_t>(cols);
+    int sms = 148;
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device);
+    const uint64_t cap = static_cast<uint64_t>(sms) * 16;
+    if (cfg->granularity == ECO_SCALE_PER_TENSOR) {
+        uint32_t* scratch = nullptr;
+        ECO_CUDA(nullptr, cudaMallocAsync(&scratch, sizeof(uint32_t), stream));
+        ECO_CUDA(nullptr, cudaMemsetAsync(scratch, 0, sizeof(uint32_t), stream));
+        const uint32_t grid = static_cast<uint32_t>(std::min<uint64_t>(cap, (numel + 1023) / 1024));
+        ECO_CUDA(nullptr, eco::launch_quantize(lc, x, static_cast<uint8_t*>(w), scale, rows, static_cast<uint32_t>(cols), 0, P, tensor_id, scratch, grid, stream));
+        ECO_CUDA(nullptr, eco::launch_quantize(lc, x, static_cast<uint8_t*>(w), scale, rows, static_cast<uint32_t>(cols), 1, P, tensor_id, scratch, grid, stream));
+        ECO_CUDA(nullptr, cudaFreeAsync(scratch, stream));
+    } else if (cfg->granularity == ECO_SCALE_PER_ROW) {
+        const uint32_t grid = static_cast<uint32_t>(std::min<uint64_t>(cap, static_cast<uint64_t>(rows)));
+        ECO_CUDA(nullptr, eco::launch_quantize(lc, x, static_cast<uint8_t*>(w), scale, rows, static_cast<uint32_t>(cols), 2, P, tensor_id, nullptr, grid, stream));
+    } else {
+        const uint64_t n_blocks = static_cast<uint64_t>(rows) * static_cast<uint64_t>((cols + 127) / 128);
+        const uint32_t grid = static_cast<uint32_t>(std::min<uint64_t>(cap, (n_blocks + 7) / 8));
+        ECO_CUDA(nullptr, eco::launch_quantize(lc, x, static_cast<uint8_t*>(w), scale, rows, static_cast<uint32_t>(cols), 3, P, tensor_id, nullptr, grid, stream));
+    }
+    return ECO_OK;
+}
+
+eco_status eco_step_host(const eco_config* cfg, const eco_tensor* tensors, size_t n, int device,
+                         float lr, float beta1, float beta2, float eps, uint64_t step, uint64_t seed,
+                         uint64_t* h2d_bytes, uint64_t* d2h_bytes) {
+    if (eco_status st = check_config(cfg, true)) return st;
+    if (!tensors || n == 0) return fail(nullptr, ECO_ERR_INVALID_ARG, "empty tensor list");
+    if (eco_status st = check_hyper(nullptr, *cfg, lr, beta1, beta2, eps, step)) return st;
+    const bool adam = cfg->optimizer == ECO_OPT_ADAM;
+    for (size_t i = 0; i < n; ++i) {
+        const eco_tensor& t = tensors[i];
+        if (eco_status st = check_shape(*cfg, t.rows, t.cols, i)) return st;
+        if (!t.w || !t.scale || !t.grad || !t.m || (adam && !t.v) || (!adam && t.v))
+            return fail(nullptr, ECO_ERR_INVALID_ARG, "tensor %zu: NULL buffer (or v given for SGDM)", i);
+    }
+    ECO_CUDA(nullptr, cudaSetDevice(device));
+
+    // Device staging: one arena, every buffer 256-byte aligned.
+    auto align = [](uint64_t x) { return (x + 255) & ~uint64_t(255); };
+    struct Stage { uint64_t w, scale, grad, m, v, wb, sb, gb, mb; };
+    std::vector<Stage> st(n);
+    uint64_t total = 0;
+    for (size_t i = 0; i < n; ++i) {
+        const uint64_t numel = static_cast<uint64_t>(tensors[i].rows) * static_cast<uint64_t>(tensors[i].cols);
+        Stage& s = st[i];
+        s.wb = code_bytes(*cfg, numel); s.sb = scale_bytes(*cfg, tensors[i].rows, tensors[i].cols);
+        s.gb = numel * 2; s.mb = numel * 4;
+        s.w = total; total += align(s.wb);
+        s.scale = total; total += align(s.sb);
+        s.grad = total; total += align(s.gb);
+        s.m = total; total += align(s.mb);
+        s.v = total; if (adam) total += align(s.mb);
+    }
+    uint8_t* arena = nullptr;
+    ECO_CUDA(nullptr, cudaMalloc(&arena, total));
+    cudaStream_t stream = nullptr;
+    eco_ctx* ctx = nullptr;
+    eco_status rc = ECO_OK;
+    uint64_t up = 0, down = 0;
+    std::vector<eco_tensor> dev(n);
+    auto bail = [&](eco_status s) {
+        if (ctx) eco_destroy(ctx);
+        if (stream) cudaStreamDestroy(stream);
+        cudaFree(arena);
+        return s;
+    };
+#define ECO_CUDA_H(call)                                                                             \
+    do {                                                                                             \
+        cudaError_t e_ = (call);                                                                     \
+        if (e_ != cudaSuccess) return bail(fail(nullptr, ECO_ERR_CUDA, "%s failed: %s", #call, cudaGetErrorString(e_))); \
+    } while (0)
+    ECO_CUDA_H(cudaStreamCreateWithFlags(&stream, cudaStreamNonBlocking));
+    for (size_t i = 0; i < n; ++i) {
+        const Stage& s = st[i];
+        dev[i] = tensors[i];
+        dev[i].w = arena + s.w;
+        dev[i].scale = arena + s.scale;
+        dev[i].grad = arena + s.grad;
+        dev[i].m = reinterpret_cast<float*>(arena + s.m);
+        dev[i].v = adam ? reinterpret_cast<float*>(arena + s.v) : nullptr;
+        ECO_CUDA_H(cudaMemcpyAsync(dev[i].w, tensors[i].w, s.wb, cudaMemcpyHostToDevice, stream));
+        ECO_CUDA_H(cudaMemcpyAsync(dev[i].scale, tensors[i].scale, s.sb, cudaMemcpyHostToDevice, stream));
+        ECO_CUDA_H(cudaMemcpyAsync(const_cast<void*>(dev[i].grad), tensors[i].grad, s.gb, cudaMemcpyHostToDevice, stream));
+        ECO_CUDA_H(cudaMemcpyAsync(dev[i].m, tensors[i].m, s.mb, cudaMemcpyHostToDevice, stream));
+        up += s.wb + s.sb + s.gb + s.mb;
+        if (adam) { ECO_CUDA_H(cudaMemcpyAsync(dev[i].v, tensors[i].v, s.mb, cudaMemcpyHostToDevice, stream)); up += s.mb; }
+    }
+    rc = eco_create(&ctx, cfg, dev.data(), n, device);
+    if (rc != ECO_OK) return bail(rc);
+    rc = eco_step(ctx, lr, beta1, beta2, eps, step, seed, stream);
+    if (rc != ECO_OK) { g_thread_error = ctx->err; return bail(rc); }
+    for (size_t i = 0; i < n; ++i) {
+        const Stage& s = st[i];
+        ECO_CUDA_H(cudaMemcpyAsync(tensors[i].w, dev[i].w, s.wb, cudaMemcpyDeviceToHost, stream));
+        ECO_CUDA_H(cudaMemcpyAsync(tensors[i].scale, dev[i].scale, s.sb, cudaMemcpyDeviceToHost, stream));
+        ECO_CUDA_H(cudaMemcpyAsync(tensors[i].m, dev[i].m, s.mb, cudaMemcpyDeviceToHost, stream));
+        down += s.wb + s.sb + s.mb;
+        if (adam) { ECO_CUDA_H(cudaMemcpyAsync(tensors[i].v, dev[i].v, s.mb, cudaMemcpyDeviceToHost, stream)); down += s.mb; }
+    }
+    ECO_CUDA_H(cudaStreamSynchronize(stream));
+#undef ECO_CUDA_H
+    if (h2d_bytes) *h2d_bytes = up;
+    if (d2h_bytes) *d2h_bytes = down;
+    return bail(ECO_OK);
+}
+
+}  // extern "C"

@@ -1,0 +1,37 @@
+// Host-side interface between the C-ABI layer (eco_api.cu) and the kernel
+// launchers (eco_kernels.cu).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "eco_device.cuh"
+
+namespace eco {
+
+struct LaunchConfig {
+    int format;      // FMT_*
+    int optimizer;   // OPT_*
+    int rounding;    // RND_*
+    int bf16_scale;  // 0: f32 scales, 1: bf16 scales
+};
+
+// Rows of 128 elements that one CTA (work unit) covers.
+int rows_per_unit();
+
+cudaError_t launch_block128(const LaunchConfig& c, const TensorDesc* descs, const uint32_t* unit_tensor,
+                            uint32_t n_units, bool generic, const StepParams& P, cudaStream_t stream);
+cudaError_t launch_tensor_amax(const LaunchConfig& c, const TensorDesc* descs, const uint32_t* unit_tensor,
+                               uint32_t n_units, const StepParams& P, uint32_t* scratch_amax, float* scratch_s_old,
+                               cudaStream_t stream);
+cudaError_t launch_tensor_apply(const LaunchConfig& c, const TensorDesc* descs, const uint32_t* unit_tensor,
+                                uint32_t n_units, const StepParams& P, const uint32_t* scratch_amax,
+                                uint32_t* scratch_amax_next, const float* scratch_s_old, bool reverse,
+                                cudaStream_t stream);
+cudaError_t launch_row(const LaunchConfig& c, const TensorDesc* descs, const uint32_t* unit_tensor,
+                       uint32_t n_units, const StepParams& P, cudaStream_t stream);
+cudaError_t launch_quantize(const LaunchConfig& c, const float* x, uint8_t* w, void* scale, uint64_t rows,
+                            uint32_t cols, int mode, const StepParams& P, uint32_t tensor_id,
+                            uint32_t* scratch_amax, uint32_t grid, cudaStream_t stream);
+
+}  // namespace eco

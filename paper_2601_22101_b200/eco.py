@@ -1,0 +1,195 @@
+"""Thin Python binding of the C-ABI in ``include/eco.h``: argument marshalling only.
+
+Every step of the ECO update runs in the CUDA kernels of ``libeco_b200.so``;
+PyTorch is used for device memory and streams.  There is no CPU fallback: if
+the shared library is missing or no CUDA device is present the calls raise.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from dataclasses import dataclass
+from typing import Optional, Sequence
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_LIB_PATH = os.path.join(_HERE, "libeco_b200.so")
+
+# enum values of include/eco.h
+ECO_OK = 0
+ECO_ERR_INVALID_ARG, ECO_ERR_UNSUPPORTED, ECO_ERR_ALIGNMENT, ECO_ERR_CUDA, ECO_ERR_NOMEM, ECO_ERR_TIMEOUT = 1, 2, 3, 4, 5, 6
+ECO_FORMAT_FP8_E4M3, ECO_FORMAT_INT4 = 0, 1
+ECO_SCALE_PER_TENSOR, ECO_SCALE_PER_ROW, ECO_SCALE_PER_BLOCK = 0, 1, 2
+ECO_SCALE_F32, ECO_SCALE_BF16 = 0, 1
+ECO_OPT_SGDM, ECO_OPT_ADAM = 0, 1
+ECO_ROUND_NEAREST, ECO_ROUND_STOCHASTIC = 0, 1
+ECO_INJECT_NONE, ECO_INJECT_ECO = 0, 1
+
+EXPORTED = ("eco_create", "eco_step", "eco_step_host", "eco_destroy", "eco_last_error", "eco_quantize",
+            "eco_set_option", "eco_num_launches", "eco_version")
+
+
+class EcoError(RuntimeError):
+    def __init__(self, status: int, message: str):
+        super().__init__(f"eco status {status}: {message}")
+        self.status = status
+
+
+class eco_config(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int32) for n in ("format", "granularity", "block", "scale_dtype", "optimizer",
+                                              "rounding", "injection", "reserved")]
+
+
+class eco_tensor(ctypes.Structure):
+    _fields_ = [("w", ctypes.c_void_p), ("scale", ctypes.c_void_p), ("grad", ctypes.c_void_p),
+                ("m", ctypes.c_void_p), ("v", ctypes.c_void_p),
+                ("rows", ctypes.c_int64), ("cols", ctypes.c_int64),
+                ("tensor_id", ctypes.c_uint32), ("reserved", ctypes.c_uint32)]
+
+
+_lib = None
+
+
+def load_library() -> ctypes.CDLL:
+    """Load ``libeco_b200.so`` (built in-tree by ``build.py``).  Fails loudly if it is absent."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(_LIB_PATH):
+            raise ImportError(f"{_LIB_PATH} is missing: run `python -m paper_2601_22101_b200.build` "
+                              "(there is no CPU fallback)")
+        L = ctypes.CDLL(_LIB_PATH)
+        vp, u64, u32, i64, f32 = ctypes.c_void_p, ctypes.c_uint64, ctypes.c_uint32, ctypes.c_int64, ctypes.c_float
+        L.eco_create.restype = ctypes.c_int
+        L.eco_create.argtypes = [ctypes.POINTER(vp), ctypes.POINTER(eco_config), ctypes.POINTER(eco_tensor),
+                                 ctypes.c_size_t, ctypes.c_int]
+        L.eco_step.restype = ctypes.c_int
+        L.eco_step.argtypes = [vp, f32, f32, f32, f32, u64, u64, vp]
+        L.eco_step_host.restype = ctypes.c_int
+        L.eco_step_host.argtypes = [ctypes.POINTER(eco_config), ctypes.POINTER(eco_tensor), ctypes.c_size_t,
+                                    ctypes.c_int, f32, f32, f32, f32, u64, u64,
+                                    ctypes.POINTER(u64), ctypes.POINTER(u64)]
+        L.eco_destroy.restype = ctypes.c_int
+        L.eco_destroy.argtypes = [vp]
+        L.eco_last_error.restype = ctypes.c_char_p
+        L.eco_last_error.argtypes = [vp]
+        L.eco_quantize.restype = ctypes.c_int
+        L.eco_quantize.argtypes = [ctypes.POINTER(eco_config), vp, i64, i64, vp, vp, u64, u64, u32, ctypes.c_int, vp]
+        L.eco_set_option.restype = ctypes.c_int
+        L.eco_set_option.argtypes = [ctypes.c_char_p, i64]
+        L.eco_num_launches.restype = ctypes.c_int
+        L.eco_num_launches.argtypes = [vp]
+        L.eco_version.restype = ctypes.c_char_p
+        _lib = L
+    return _lib
+
+
+@dataclass
+class Config:
+    format: int = ECO_FORMAT_FP8_E4M3
+    granularity: int = ECO_SCALE_PER_BLOCK
+    block: int = 128
+    scale_dtype: int = ECO_SCALE_F32
+    optimizer: int = ECO_OPT_ADAM
+    rounding: int = ECO_ROUND_STOCHASTIC
+    injection: int = ECO_INJECT_ECO
+
+    def c(self) -> eco_config:
+        return eco_config(self.format, self.granularity, self.block, self.scale_dtype, self.optimizer,
+                          self.rounding, self.injection, 0)
+
+
+@dataclass
+class Tensor:
+    """Device buffers of one parameter (torch CUDA tensors) or, for ``eco_step_host``, host
+    buffers (torch CPU tensors or numpy arrays)."""
+    w: object
+    scale: object
+    grad: object
+    m: object
+    v: Optional[object]
+    rows: int
+    cols: int
+    tensor_id: int
+
+
+def _addr(x) -> Optional[int]:
+    if x is None:
+        return None
+    if hasattr(x, "data_ptr"):
+        assert x.is_contiguous(), "buffers must be contiguous"
+        return x.data_ptr()
+    return x.ctypes.data   # numpy
+
+
+def _raise(status: int, handle=None):
+    msg = load_library().eco_last_error(handle)
+    raise EcoError(status, msg.decode() if msg else "")
+
+
+def _tensor_array(tensors: Sequence[Tensor]):
+    arr = (eco_tensor * len(tensors))()
+    for i, t in enumerate(tensors):
+        arr[i] = eco_tensor(_addr(t.w), _addr(t.scale), _addr(t.grad), _addr(t.m), _addr(t.v),
+                            t.rows, t.cols, t.tensor_id, 0)
+    return arr
+
+
+def eco_create(cfg: Config, tensors: Sequence[Tensor], device: int = 0) -> int:
+    """Bind a tensor list; returns the context handle.  See ``eco_create`` in include/eco.h."""
+    L = load_library()
+    handle = ctypes.c_void_p()
+    c = cfg.c()
+    arr = _tensor_array(tensors)
+    st = L.eco_create(ctypes.byref(handle), ctypes.byref(c), arr, len(tensors), device)
+    if st != ECO_OK:
+        _raise(st)
+    return handle.value
+
+
+def eco_step(handle: int, lr: float, beta1: float, beta2: float, eps: float, step: int, seed: int,
+             stream: int = 0) -> None:
+    """Enqueue one ECO step on ``stream`` (a raw cudaStream_t).  See ``eco_step`` in include/eco.h."""
+    st = load_library().eco_step(handle, lr, beta1, beta2, eps, step, seed, stream)
+    if st != ECO_OK:
+        _raise(st, handle)
+
+
+def eco_step_host(cfg: Config, tensors: Sequence[Tensor], lr: float, beta1: float, beta2: float, eps: float,
+                  step: int, seed: int, device: int = 0):
+    """One step on state held in host memory; returns (h2d_bytes, d2h_bytes)."""
+    L = load_library()
+    c = cfg.c()
+    arr = _tensor_array(tensors)
+    up, down = ctypes.c_uint64(), ctypes.c_uint64()
+    st = L.eco_step_host(ctypes.byref(c), arr, len(tensors), device, lr, beta1, beta2, eps, step, seed,
+                         ctypes.byref(up), ctypes.byref(down))
+    if st != ECO_OK:
+        _raise(st)
+    return up.value, down.value
+
+
+def eco_destroy(handle: int) -> None:
+    load_library().eco_destroy(handle)
+
+
+def eco_quantize(cfg: Config, x, rows: int, cols: int, w, scale, seed: int = 0, step: int = 0,
+                 tensor_id: int = 0, device: int = 0, stream: int = 0) -> None:
+    """theta_hat_0 = q(x) on the device.  See ``eco_quantize`` in include/eco.h."""
+    c = cfg.c()
+    st = load_library().eco_quantize(ctypes.byref(c), _addr(x), rows, cols, _addr(w), _addr(scale),
+                                     seed, step, tensor_id, device, stream)
+    if st != ECO_OK:
+        _raise(st)
+
+
+def eco_set_option(name: str, value: int) -> None:
+    st = load_library().eco_set_option(name.encode(), value)
+    if st != ECO_OK:
+        _raise(st)
+
+
+def eco_num_launches(handle: int) -> int:
+    return load_library().eco_num_launches(handle)
+
+
+def eco_version() -> str:
+    return load_library().eco_version().decode()

@@ -1,0 +1,179 @@
+"""GPU parity: the CUDA path (through the C-ABI) against the CPU oracle on the same seeded inputs.
+Bar: quantized codes and scales bit-exact; FP32 moments within 1e-6 relative / 1e-7 absolute."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from oracle_runner import OracleState, oracle_config
+from paper_2601_22101_b200 import eco, workloads as wl
+from paper_2601_22101_b200.state import DeviceState, config_of
+
+pytestmark = pytest.mark.gpu
+
+RTOL, ATOL = 1e-6, 1e-7
+
+
+def _np(t):
+    return t.detach().cpu().numpy()
+
+
+def _scale_bits(t):
+    t = t.detach().cpu()
+    return (t.view(torch.int16) if t.dtype == torch.bfloat16 else t.view(torch.int32)).numpy()
+
+
+def _oracle_scale_bits(s):
+    return s.view(np.int16) if s.dtype == np.uint16 else s.view(np.int32)
+
+
+def compare(dev: DeviceState, ora: OracleState, where=""):
+    for i, t in enumerate(dev.workload.tensors):
+        d = dev.tensors[i]
+        tag = f"{where} tensor {i} {t.name} [{t.rows}x{t.cols}]"
+        codes = _np(d.w)
+        bad = np.nonzero(codes != ora.w[i])[0]
+        assert bad.size == 0, f"{tag}: {bad.size} code mismatches, first at byte {bad[:5]}: gpu {codes[bad[:5]]} oracle {ora.w[i][bad[:5]]}"
+        assert (_scale_bits(d.scale) == _oracle_scale_bits(ora.scale[i])).all(), f"{tag}: scales differ"
+        np.testing.assert_allclose(_np(d.m), ora.m[i], rtol=RTOL, atol=ATOL, err_msg=tag + " m")
+        if ora.v[i] is not None:
+            np.testing.assert_allclose(_np(d.v), ora.v[i], rtol=RTOL, atol=ATOL, err_msg=tag + " v")
+
+
+def run_chained(w: wl.Workload, steps: int, check_every: int = 1, injection=eco.ECO_INJECT_ECO):
+    dev = DeviceState(w)
+    dev.init_from_host()
+    ora = OracleState(w, injection=oracle.INJECT_ECO if injection == eco.ECO_INJECT_ECO else oracle.INJECT_NONE)
+    compare(dev, ora, "init")
+    dev.create(injection)
+    try:
+        for step in range(1, steps + 1):
+            grads = [wl.gradient_bf16(w, t, step) for t in w.tensors]
+            for i, g in enumerate(grads):
+                dev.tensors[i].grad.view(torch.int16).copy_(torch.from_numpy(g.view(np.int16)))
+            dev.step(step)
+            ora.step(step, grads)
+            if step % check_every == 0 or step == steps:
+                torch.cuda.synchronize()
+                compare(dev, ora, f"step {step}")
+    finally:
+        dev.destroy()
+    return dev, ora
+
+
+def _mini(fmt, gran, sdt, opt, rnd, shapes, lr=1e-3, grad_std=1e-3):
+    ts = [wl.TensorSpec(f"t{i}", r, c, 100 + 7 * i, zero_grad=(i == 1 and len(shapes) > 2)) for i, (r, c) in enumerate(shapes)]
+    return wl.Workload("mini", fmt, gran, 128, sdt, opt, rnd, lr=lr, beta1=0.9, beta2=0.95, eps=1e-8,
+                       weight_std=0.02, grad_std=grad_std, steps=6, step_seed=0xABCDEF0123, tensors=ts)
+
+
+RAGGED = [(3, 384), (2, 4224), (5, 200), (1, 2), (7, 130), (33, 1024), (1, 8190), (4, 126)]
+RAGGED_FP8_ONLY = [(1, 1), (3, 127), (2, 129), (5, 333)]
+
+
+@pytest.mark.parametrize("gran", [wl.PER_BLOCK, wl.PER_TENSOR, wl.PER_ROW])
+@pytest.mark.parametrize("opt", [wl.SGDM, wl.ADAM])
+@pytest.mark.parametrize("rnd", [wl.RTN, wl.SR])
+@pytest.mark.parametrize("fmt,sdt", [(wl.FP8_E4M3, wl.SCALE_F32), (wl.FP8_E4M3, wl.SCALE_BF16),
+                                     (wl.INT4, wl.SCALE_BF16), (wl.INT4, wl.SCALE_F32)])
+def test_step_parity_ragged_shapes(fmt, sdt, opt, rnd, gran):
+    shapes = RAGGED + (RAGGED_FP8_ONLY if fmt == wl.FP8_E4M3 else [])
+    run_chained(_mini(fmt, gran, sdt, opt, rnd, shapes), steps=6)
+
+
+@pytest.mark.parametrize("fmt", [wl.FP8_E4M3, wl.INT4])
+@pytest.mark.parametrize("gran", [wl.PER_BLOCK, wl.PER_TENSOR, wl.PER_ROW])
+@pytest.mark.parametrize("rnd", [wl.RTN, wl.SR])
+def test_quantize_parity(fmt, gran, rnd):
+    """eco_quantize against the oracle's q(x), including stochastic rounding."""
+    rng = np.random.default_rng(21)
+    w = _mini(fmt, gran, wl.SCALE_F32, wl.SGDM, rnd, RAGGED + (RAGGED_FP8_ONLY if fmt == wl.FP8_E4M3 else []))
+    cfg_o = oracle_config(w)
+    cfg_d = config_of(w)
+    for t in w.tensors:
+        x = (rng.standard_normal((t.rows, t.cols)) * 0.02).astype(np.float32)
+        x.flat[:: 17] = 0.0
+        x.flat[:: 29] *= 1e-4          # exercise the subnormal range of the grid
+        ow, os_ = oracle.quantize(cfg_o, x, seed=99, step=3, tensor_id=t.tensor_id)
+        dx = torch.from_numpy(x).cuda()
+        dw = torch.zeros(w.code_bytes(t), dtype=torch.uint8, device="cuda")
+        ds = torch.zeros(w.n_scales(t), dtype=torch.float32, device="cuda")
+        eco.eco_quantize(cfg_d, dx, t.rows, t.cols, dw, ds, seed=99, step=3, tensor_id=t.tensor_id)
+        torch.cuda.synchronize()
+        assert (_np(dw) == ow).all(), (t.rows, t.cols)
+        assert (_np(ds).view(np.int32) == os_.view(np.int32)).all()
+
+
+def test_zero_and_tiny_blocks():
+    """Degenerate cases: all-zero tensors (scale 1, zero codes), zero gradients, tiny values."""
+    w = _mini(wl.FP8_E4M3, wl.PER_BLOCK, wl.SCALE_F32, wl.ADAM, wl.SR, [(2, 256), (1, 128), (3, 200)])
+    zero_w = [np.zeros((t.rows, t.cols), np.float32) for t in w.tensors]
+    zero_w[2][:] = 1e-30
+    dev = DeviceState(w)
+    for i, x in enumerate(zero_w):
+        dev.quantize_from(i, torch.from_numpy(x).cuda())
+    ora = OracleState(w, weights=zero_w)
+    compare(dev, ora, "init")
+    assert (_np(dev.tensors[0].scale) == 1.0).all() and (_np(dev.tensors[0].w) == 0).all()
+    dev.create()
+    try:
+        for step in (1, 2, 3):
+            grads = [np.zeros(t.numel, np.uint16) if step < 3 else wl.gradient_bf16(w, t, step) for t in w.tensors]
+            for i, g in enumerate(grads):
+                dev.tensors[i].grad.view(torch.int16).copy_(torch.from_numpy(g.view(np.int16)))
+            dev.step(step)
+            ora.step(step, grads)
+            torch.cuda.synchronize()
+            compare(dev, ora, f"step {step}")
+    finally:
+        dev.destroy()
+
+
+@pytest.mark.parametrize("rnd", [wl.RTN, wl.SR])
+def test_c1_linear_10_steps(rnd):
+    run_chained(wl.c1(rnd), steps=10)
+
+
+def test_naive_removal_flag_matches_oracle():
+    """Injection switched off (the naive regime of Sec. 3.4) on the same kernel."""
+    w = _mini(wl.FP8_E4M3, wl.PER_BLOCK, wl.SCALE_F32, wl.SGDM, wl.SR, [(4, 512), (3, 200)])
+    run_chained(w, steps=4, injection=eco.ECO_INJECT_NONE)
+
+
+def test_c2_decoder_100_chained_steps_full_size():
+    run_chained(wl.c2(), steps=100, check_every=25)
+
+
+def test_c3_slice_100_chained_steps():
+    run_chained(wl.shape_slice(wl.c3(), max_rows=1024), steps=100, check_every=50)
+
+
+def test_c4_slice_100_chained_steps():
+    run_chained(wl.shape_slice(wl.c4(layers=2, experts=4)), steps=100, check_every=50)
+
+
+def test_c5_slice_100_chained_steps():
+    run_chained(wl.shape_slice(wl.c5(), max_rows=512), steps=100, check_every=50)
+
+
+def test_checkpoint_resume_is_bit_exact():
+    """State = (codes, scales, m, v) + (step, seed): 6 steps straight equal 3 + reload + 3."""
+    w = _mini(wl.FP8_E4M3, wl.PER_TENSOR, wl.SCALE_F32, wl.ADAM, wl.SR, [(8, 640), (3, 200)])
+    a = DeviceState(w); a.init_from_host(); a.create()
+    b = DeviceState(w); b.init_from_host(); b.create()
+    for step in range(1, 7):
+        a.set_grads_from_host(step); a.step(step)
+        b.set_grads_from_host(step); b.step(step)
+        if step == 3:
+            torch.cuda.synchronize()
+            saved = [(t.w.clone(), t.scale.clone(), t.m.clone(), t.v.clone()) for t in b.tensors]
+            b.destroy()
+            b = DeviceState(w)
+            for t, s in zip(b.tensors, saved):
+                t.w.copy_(s[0]); t.scale.copy_(s[1]); t.m.copy_(s[2]); t.v.copy_(s[3])
+            b.create()
+    torch.cuda.synchronize()
+    for ta, tb in zip(a.tensors, b.tensors):
+        assert torch.equal(ta.w, tb.w) and torch.equal(ta.scale, tb.scale)
+        assert torch.equal(ta.m, tb.m) and torch.equal(ta.v, tb.v)
+    a.destroy(); b.destroy()
