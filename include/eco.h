@@ -33,7 +33,7 @@ typedef enum eco_status {
     ECO_ERR_ALIGNMENT = 3,   /* a buffer is not 16-byte aligned */
     ECO_ERR_CUDA = 4,        /* a CUDA runtime call failed; eco_last_error has its text */
     ECO_ERR_NOMEM = 5,
-    ECO_ERR_TIMEOUT = 6      /* reserved for bounded device-side waits */
+    ECO_ERR_TIMEOUT = 6      /* a bounded device-side wait expired (see eco_check) */
 } eco_status;
 
 /* Weight format (Sec. 3.1; rho = largest representable magnitude). */
@@ -141,6 +141,15 @@ eco_status eco_step_host(const eco_config* cfg, const eco_tensor* tensors, size_
                          float lr, float beta1, float beta2, float eps, uint64_t step, uint64_t seed,
                          uint64_t* h2d_bytes, uint64_t* d2h_bytes);
 
+/*
+ * eco_check -- synchronize cuda_stream and report whether any kernel of this context gave up on a
+ * device-side wait.  The streaming kernels wait on shared-memory barriers for their asynchronous
+ * copies; every such wait is bounded (about two seconds of clock cycles), after which the kernel
+ * records a code in the context and exits instead of hanging.
+ * Returns ECO_OK, ECO_ERR_TIMEOUT (state of the tensors is then undefined), or ECO_ERR_CUDA.
+ */
+eco_status eco_check(eco_ctx* ctx, void* cuda_stream);
+
 /* eco_destroy -- free the context's tables and scratch (synchronizes the device). NULL is allowed. */
 eco_status eco_destroy(eco_ctx* ctx);
 
@@ -172,6 +181,10 @@ eco_status eco_quantize(const eco_config* cfg, const float* x, int64_t rows, int
  *                     default; 0 = one pair for the whole context)
  *   "reverse_pass2"   per-tensor scales only: 1 (default) walks pass 2 in the opposite order
  *                     of pass 1 so that it starts with the most recently read data
+ *   "use_stream"      1 (default) uses the persistent kernels fed by bulk asynchronous copies
+ *                     wherever a tensor consists of whole, aligned 128-element rows; 0 forces
+ *                     the direct-load kernels everywhere
+ *   "ctas_per_sm"     persistent grid size in CTAs per SM, 1 or 2 (default 2)
  * No option changes any result bit.  Errors: ECO_ERR_INVALID_ARG for an unknown name.
  */
 eco_status eco_set_option(const char* name, int64_t value);

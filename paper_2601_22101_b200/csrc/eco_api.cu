@@ -22,7 +22,7 @@ namespace {
 
 thread_local std::string g_thread_error;
 
-enum LaunchKind { KIND_BLOCK_FAST = 0, KIND_BLOCK_GENERIC = 1, KIND_TENSOR = 2, KIND_ROW = 3 };
+enum LaunchKind { KIND_BLOCK_FAST = 0, KIND_BLOCK_GENERIC = 1, KIND_TENSOR = 2, KIND_ROW = 3, KIND_TENSOR_STREAM = 4 };
 
 struct Launch {
     int kind;
@@ -35,6 +35,8 @@ struct Launch {
 struct Options {
     int64_t l2_group_bytes = -1;   // per-tensor scale: input bytes per launch pair; -1 = half of the L2 size, 0 = one group
     int64_t reverse_pass2 = 1;     // per-tensor scale: walk pass 2 in the opposite order of pass 1
+    int64_t use_stream = 1;        // 1: TMA-fed persistent kernels where the layout allows; 0: direct-load kernels only
+    int64_t ctas_per_sm = 2;       // persistent grid = ctas_per_sm * SM count
 };
 Options g_options;
 
@@ -49,6 +51,8 @@ struct eco_ctx {
     uint32_t* d_unit_tensor = nullptr;
     uint32_t* d_amax[2] = {nullptr, nullptr};
     float* d_s_old = nullptr;
+    uint32_t* d_status = nullptr;
+    int grid_cap = 296;
     uint64_t calls = 0;
     bool reverse_pass2 = true;
     int num_launches = 0;
@@ -186,6 +190,10 @@ StepParams derive_params(const eco_config& cfg, float lr_f, float beta1_f, float
     P.step_lo = static_cast<uint32_t>(step);
     P.step_hi = static_cast<uint32_t>(step >> 32);
     P.inject = cfg.injection == ECO_INJECT_ECO ? 1 : 0;
+    for (uint32_t r = 0; r < 10; ++r) {
+        P.rk0[r] = P.seed_lo + r * 0x9E3779B9u;
+        P.rk1[r] = P.seed_hi + r * 0xBB67AE85u;
+    }
     return P;
 }
 
@@ -207,6 +215,12 @@ eco_status eco_set_option(const char* name, int64_t value) {
     if (!name) return fail(nullptr, ECO_ERR_INVALID_ARG, "option name is NULL");
     if (!std::strcmp(name, "l2_group_bytes")) { g_options.l2_group_bytes = value; return ECO_OK; }
     if (!std::strcmp(name, "reverse_pass2")) { g_options.reverse_pass2 = value; return ECO_OK; }
+    if (!std::strcmp(name, "use_stream")) { g_options.use_stream = value; return ECO_OK; }
+    if (!std::strcmp(name, "ctas_per_sm")) {
+        if (value < 1 || value > 2) return fail(nullptr, ECO_ERR_INVALID_ARG, "ctas_per_sm must be 1 or 2");
+        g_options.ctas_per_sm = value;
+        return ECO_OK;
+    }
     return fail(nullptr, ECO_ERR_INVALID_ARG, "unknown option '%s'", name);
 }
 
@@ -256,6 +270,8 @@ eco_status eco_create(eco_ctx** out, const eco_config* cfg, const eco_tensor* te
     ctx->device = device;
     ctx->lc = launch_config(*cfg);
     ctx->reverse_pass2 = g_options.reverse_pass2 != 0;
+    ctx->grid_cap = static_cast<int>(g_options.ctas_per_sm) * prop.multiProcessorCount;
+    const bool use_stream = g_options.use_stream != 0;
 
     // ---- work-unit tables -------------------------------------------------
     const uint64_t rpu = static_cast<uint64_t>(eco::rows_per_unit());
@@ -292,7 +308,7 @@ eco_status eco_create(eco_ctx** out, const eco_config* cfg, const eco_tensor* te
                 d.n_blocks = static_cast<uint64_t>(tensors[members[k]].rows);
                 nu = d.n_blocks;
             } else {
-                d.n_blocks = (kind == KIND_TENSOR) ? (d.numel + 127) / 128
+                d.n_blocks = (kind == KIND_TENSOR || kind == KIND_TENSOR_STREAM) ? (d.numel + 127) / 128
                                                    : static_cast<uint64_t>(tensors[members[k]].rows) * d.blocks_per_row;
                 nu = (d.n_blocks + rpu - 1) / rpu;
             }
@@ -310,7 +326,7 @@ eco_status eco_create(eco_ctx** out, const eco_config* cfg, const eco_tensor* te
     bool ok = true;
     if (cfg->granularity == ECO_SCALE_PER_BLOCK) {
         std::vector<size_t> fast, generic;
-        for (size_t i = 0; i < n; ++i) ((tensors[i].cols % 128 == 0) ? fast : generic).push_back(i);
+        for (size_t i = 0; i < n; ++i) ((use_stream && tensors[i].cols % 128 == 0) ? fast : generic).push_back(i);
         ok = add_launch(KIND_BLOCK_FAST, fast) && add_launch(KIND_BLOCK_GENERIC, generic);
         ctx->num_launches = static_cast<int>(ctx->launches.size());
     } else if (cfg->granularity == ECO_SCALE_PER_ROW) {
@@ -326,17 +342,26 @@ eco_status eco_create(eco_ctx** out, const eco_config* cfg, const eco_tensor* te
         const double in_bytes_per_elem = (cfg->format == ECO_FORMAT_FP8_E4M3 ? 1.0 : 0.5) + 2.0 + (adam ? 8.0 : 4.0);
         std::vector<size_t> group;
         double group_bytes = 0;
+        // tensors made of whole 128-element rows go to the streaming kernels, the rest to the direct-load ones
+        auto flush_group = [&]() {
+            std::vector<size_t> fast, generic;
+            for (size_t i : group) {
+                const uint64_t numel = static_cast<uint64_t>(tensors[i].rows) * static_cast<uint64_t>(tensors[i].cols);
+                ((use_stream && numel % 128 == 0) ? fast : generic).push_back(i);
+            }
+            return add_launch(KIND_TENSOR_STREAM, fast) && add_launch(KIND_TENSOR, generic);
+        };
         for (size_t i = 0; i < n && ok; ++i) {
             const double b = in_bytes_per_elem * static_cast<double>(tensors[i].rows) * static_cast<double>(tensors[i].cols);
             if (!group.empty() && budget > 0 && group_bytes + b > static_cast<double>(budget)) {
-                ok = add_launch(KIND_TENSOR, group);
+                ok = flush_group();
                 group.clear();
                 group_bytes = 0;
             }
             group.push_back(i);
             group_bytes += b;
         }
-        if (ok) ok = add_launch(KIND_TENSOR, group);
+        if (ok) ok = flush_group();
         ctx->num_launches = 2 * static_cast<int>(ctx->launches.size());
     }
     if (!ok) {
@@ -366,6 +391,8 @@ eco_status eco_create(eco_ctx** out, const eco_config* cfg, const eco_tensor* te
         }
         ECO_CUDA_CTX(cudaMalloc(&ctx->d_s_old, n * sizeof(float)));
     }
+    ECO_CUDA_CTX(cudaMalloc(&ctx->d_status, sizeof(uint32_t)));
+    ECO_CUDA_CTX(cudaMemset(ctx->d_status, 0, sizeof(uint32_t)));
     ECO_CUDA_CTX(cudaDeviceSynchronize());
 #undef ECO_CUDA_CTX
     *out = ctx;
@@ -384,8 +411,19 @@ eco_status eco_step(eco_ctx* ctx, float lr, float beta1, float beta2, float eps,
         const uint32_t* units = ctx->d_unit_tensor + L.unit_offset;
         switch (L.kind) {
             case KIND_BLOCK_FAST:
+                ECO_CUDA(ctx, eco::launch_stream(ctx->lc, eco::STREAM_BLOCK, descs, units, L.n_units, P, nullptr, nullptr,
+                                                 nullptr, false, ctx->d_status, ctx->grid_cap, stream));
+                break;
             case KIND_BLOCK_GENERIC:
-                ECO_CUDA(ctx, eco::launch_block128(ctx->lc, descs, units, L.n_units, L.kind == KIND_BLOCK_GENERIC, P, stream));
+                ECO_CUDA(ctx, eco::launch_block128(ctx->lc, descs, units, L.n_units, true, P, stream));
+                break;
+            case KIND_TENSOR_STREAM:
+                ECO_CUDA(ctx, eco::launch_stream(ctx->lc, eco::STREAM_TENSOR_AMAX, descs, units, L.n_units, P,
+                                                 ctx->d_amax[parity], nullptr, ctx->d_s_old, false, ctx->d_status,
+                                                 ctx->grid_cap, stream));
+                ECO_CUDA(ctx, eco::launch_stream(ctx->lc, eco::STREAM_TENSOR_APPLY, descs, units, L.n_units, P,
+                                                 ctx->d_amax[parity], ctx->d_amax[parity ^ 1], ctx->d_s_old,
+                                                 ctx->reverse_pass2, ctx->d_status, ctx->grid_cap, stream));
                 break;
             case KIND_ROW:
                 ECO_CUDA(ctx, eco::launch_row(ctx->lc, descs, units, L.n_units, P, stream));
@@ -401,6 +439,17 @@ eco_status eco_step(eco_ctx* ctx, float lr, float beta1, float beta2, float eps,
     return ECO_OK;
 }
 
+eco_status eco_check(eco_ctx* ctx, void* cuda_stream) {
+    if (!ctx) return fail(nullptr, ECO_ERR_INVALID_ARG, "ctx is NULL");
+    ECO_CUDA(ctx, cudaStreamSynchronize(static_cast<cudaStream_t>(cuda_stream)));
+    uint32_t code = 0;
+    ECO_CUDA(ctx, cudaMemcpy(&code, ctx->d_status, sizeof code, cudaMemcpyDeviceToHost));
+    if (code != 0)
+        return fail(ctx, ECO_ERR_TIMEOUT, "a bounded wait inside a kernel expired (code %u: 1 = producer waiting for a free "
+                    "stage, 2 = producer draining its copies, 3 = consumer waiting for data)", code);
+    return ECO_OK;
+}
+
 eco_status eco_destroy(eco_ctx* ctx) {
     if (!ctx) return ECO_OK;
     cudaSetDevice(ctx->device);
@@ -410,6 +459,7 @@ eco_status eco_destroy(eco_ctx* ctx) {
     cudaFree(ctx->d_amax[0]);
     cudaFree(ctx->d_amax[1]);
     cudaFree(ctx->d_s_old);
+    cudaFree(ctx->d_status);
     delete ctx;
     return ECO_OK;
 }

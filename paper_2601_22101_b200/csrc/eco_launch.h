@@ -18,6 +18,17 @@ struct LaunchConfig {
 
 // Rows of 128 elements that one CTA (work unit) covers.
 int rows_per_unit();
+int stream_unit_rows();
+
+// Modes of the TMA-fed streaming kernel (eco_stream_kernels.cu).
+enum : int { STREAM_BLOCK = 0, STREAM_TENSOR_AMAX = 1, STREAM_TENSOR_APPLY = 2 };
+enum : int { MODE_BLOCK = STREAM_BLOCK, MODE_TENSOR_AMAX = STREAM_TENSOR_AMAX, MODE_TENSOR_APPLY = STREAM_TENSOR_APPLY };
+
+// Persistent launch over n_units work units; grid = min(n_units, grid_cap).  `status` is a device word
+// that receives a non-zero code if a bounded wait inside the kernel expires.
+cudaError_t launch_stream(const LaunchConfig& c, int mode, const TensorDesc* descs, const uint32_t* unit_tensor,
+                          uint32_t n_units, const StepParams& P, uint32_t* amax, uint32_t* amax_next, float* s_old,
+                          bool reverse, uint32_t* status, int grid_cap, cudaStream_t stream);
 
 cudaError_t launch_block128(const LaunchConfig& c, const TensorDesc* descs, const uint32_t* unit_tensor,
                             uint32_t n_units, bool generic, const StepParams& P, cudaStream_t stream);

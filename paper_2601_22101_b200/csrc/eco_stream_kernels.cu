@@ -1,0 +1,361 @@
+// Streaming kernels of the ECO step for sm_100a: persistent CTAs fed by the TMA
+// engine.
+//
+// One CTA = 1 producer warp + 8 consumer warps, two CTAs per SM.  The parameter
+// set is cut into units of 32 rows of 128 elements (4096 parameters); each CTA
+// owns a contiguous range of units.  For every unit the producer issues one
+// bulk asynchronous copy (cp.async.bulk, global -> shared, completion counted
+// on an mbarrier) per input stream -- codes, bf16 gradient, m and, for Adam, v
+// -- into a ring of shared-memory stages, and stages the unit's old scales and
+// a small header next to them.  Consumer warps wait for the stage, pull their 4
+// rows out of shared memory with conflict-free 16-byte reads, hand the stage
+// back, and do all arithmetic from registers; results go straight to global
+// memory with coalesced 16-byte stores.  Global loads therefore cost no issue
+// slots and no registers, and the bytes in flight per SM are set by the ring
+// depth (tens of KB), not by occupancy.
+//
+// Every wait on an mbarrier is bounded: after ~2 s worth of clock cycles the
+// waiter records a code in the context's status word and leaves; the producer
+// first waits (bounded again) for the copies it has in flight.
+#include "eco_device.cuh"
+#include "eco_launch.h"
+
+namespace eco {
+
+constexpr int kConsumerWarps = 8;
+constexpr int kStreamThreads = (kConsumerWarps + 1) * 32;
+constexpr int kUnitRows = kConsumerWarps * 4;      // rows of 128 elements per unit
+constexpr long long kWaitLimitCycles = 4000000000LL;
+
+// What the producer tells the consumers about a unit.
+struct StageHeader {
+    uint8_t* w;
+    void* scale;
+    float* m;
+    float* v;
+    uint64_t row0;        // first row of the unit inside its tensor
+    uint32_t nrows;       // rows present (the last unit of a tensor may be short)
+    uint32_t tensor_id;
+    uint32_t slot;
+    float s_old;          // per-tensor modes
+    float s_new, inv_new; // per-tensor pass 2
+};
+static_assert(sizeof(StageHeader) <= 64, "header must fit its slot");
+
+template <int FMT, int OPT>
+struct StageLayout {
+    static constexpr int kCodeRow = FMT == FMT_FP8 ? 128 : 64;   // bytes of codes per row
+    static constexpr int kHeader = 0;
+    static constexpr int kScales = 128;                          // kUnitRows floats
+    static constexpr int kCodes = kScales + kUnitRows * 4;
+    static constexpr int kGrad = kCodes + kUnitRows * kCodeRow;
+    static constexpr int kM = kGrad + kUnitRows * 256;
+    static constexpr int kV = kM + kUnitRows * 512;
+    static constexpr int kBytes = kV + (OPT == OPT_ADAM ? kUnitRows * 512 : 0);
+    static constexpr int kStages = OPT == OPT_ADAM ? 2 : 3;
+    static constexpr int kBarriers = 128;                        // 2 * kStages mbarriers, padded
+    static constexpr int kSmem = kBarriers + kStages * kBytes;
+    static_assert(kBytes % 128 == 0, "stages stay 128-byte aligned");
+};
+
+// ---- mbarrier / bulk-copy primitives ----------------------------------------
+__device__ __forceinline__ uint32_t smem_addr(const void* p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("{ .reg .b64 st; mbarrier.arrive.shared::cta.b64 st, [%0]; }" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("{ .reg .b64 st; mbarrier.arrive.expect_tx.shared::cta.b64 st, [%0], %1; }" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile("{ .reg .pred p; mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2; selp.u32 %0, 1, 0, p; }"
+                 : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+// Bounded wait; on expiry records `code` and returns false.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, uint32_t* status, uint32_t code) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    while (!mbar_try_wait(bar, parity)) {
+        if (clock64() - t0 > kWaitLimitCycles) {
+            atomicExch(status, code);
+            return false;
+        }
+    }
+    return true;
+}
+// Plain (single-CTA) bulk copy global -> shared, completion on an mbarrier of this CTA.
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+
+__device__ __forceinline__ float reduce_rows4s(const float a[4], int lane) {
+    const bool b4 = lane & 16, b3 = lane & 8;
+    const float send_x = b4 ? a[0] : a[2], send_y = b4 ? a[1] : a[3];
+    const float keep_x = b4 ? a[2] : a[0], keep_y = b4 ? a[3] : a[1];
+    const float x = fmaxf(keep_x, __shfl_xor_sync(0xFFFFFFFFu, send_x, 16));
+    const float y = fmaxf(keep_y, __shfl_xor_sync(0xFFFFFFFFu, send_y, 16));
+    const float send = b3 ? x : y, keep = b3 ? y : x;
+    float z = fmaxf(keep, __shfl_xor_sync(0xFFFFFFFFu, send, 8));
+    z = fmaxf(z, __shfl_xor_sync(0xFFFFFFFFu, z, 4));
+    z = fmaxf(z, __shfl_xor_sync(0xFFFFFFFFu, z, 2));
+    z = fmaxf(z, __shfl_xor_sync(0xFFFFFFFFu, z, 1));
+    return z;
+}
+
+__device__ __forceinline__ uint32_t units_of(const TensorDesc& T) {
+    return static_cast<uint32_t>((T.n_blocks + kUnitRows - 1) / kUnitRows);
+}
+
+// ---------------------------------------------------------------------------
+// MODE_BLOCK        1x128 block scales, whole step in one pass
+// MODE_TENSOR_AMAX  per-tensor scale, pass 1: max |theta~| per tensor
+// MODE_TENSOR_APPLY per-tensor scale, pass 2: quantize with the tensor's scale
+// Tensors handled here have a whole number of 128-element rows that start on
+// 128-element boundaries (cols % 128 == 0, or a flat tensor with numel % 128 == 0).
+// ---------------------------------------------------------------------------
+template <int FMT, int OPT, int RND, int MODE>
+__global__ void __launch_bounds__(kStreamThreads, 2)
+eco_stream_kernel(const TensorDesc* __restrict__ descs, const uint32_t* __restrict__ unit_tensor,
+                  const uint32_t n_units, const StepParams P, const int bf16_scale,
+                  uint32_t* __restrict__ scratch_amax, uint32_t* __restrict__ scratch_amax_next,
+                  float* __restrict__ scratch_s_old, const int reverse, uint32_t* __restrict__ status) {
+    using SL = StageLayout<FMT, OPT>;
+    constexpr int S = SL::kStages;
+    extern __shared__ __align__(128) uint8_t smem[];
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem);
+    const uint32_t full0 = smem_addr(bars), empty0 = smem_addr(bars + S);
+    uint8_t* stage0 = smem + SL::kBarriers;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < S; ++s) {
+            mbar_init(full0 + 8 * s, 2);                 // producer: expect_tx arrival + header/scales arrival
+            mbar_init(empty0 + 8 * s, kConsumerWarps);
+        }
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+
+    const uint32_t lo = static_cast<uint32_t>(static_cast<uint64_t>(n_units) * blockIdx.x / gridDim.x);
+    const uint32_t hi = static_cast<uint32_t>(static_cast<uint64_t>(n_units) * (blockIdx.x + 1) / gridDim.x);
+    const uint32_t n_my = hi - lo;
+    if (n_my == 0) return;
+
+    if (warp == kConsumerWarps) {
+        // ------------------------------ producer ------------------------------
+        uint32_t t = __ldg(unit_tensor + (reverse ? hi - 1 : lo));
+        TensorDesc T = descs[t];
+        uint32_t issued = 0;
+        bool ok = true;
+        for (uint32_t it = 0; it < n_my && ok; ++it) {
+            const uint32_t unit = reverse ? (hi - 1 - it) : (lo + it);
+            if (!reverse) { while (unit >= T.first_unit + units_of(T)) T = descs[++t]; }
+            else          { while (unit < T.first_unit) T = descs[--t]; }
+            const uint32_t s = it % S, ph = (it / S) & 1;
+            ok = mbar_wait(empty0 + 8 * s, ph ^ 1, status, 1u);
+            if (!ok) break;
+            uint8_t* st = stage0 + static_cast<size_t>(s) * SL::kBytes;
+            const uint32_t local = unit - T.first_unit;
+            const uint64_t row0 = static_cast<uint64_t>(local) * kUnitRows;
+            const uint64_t left = T.n_blocks - row0;
+            const uint32_t nrows = left < kUnitRows ? static_cast<uint32_t>(left) : kUnitRows;
+            const uint32_t full = full0 + 8 * s;
+            if (lane == 0) {
+                const uint32_t cb = nrows * SL::kCodeRow, gb = nrows * 256u, mb = nrows * 512u;
+                mbar_arrive_expect_tx(full, cb + gb + mb + (OPT == OPT_ADAM ? mb : 0u));
+                bulk_load(smem_addr(st + SL::kCodes), T.w + row0 * SL::kCodeRow, cb, full);
+                bulk_load(smem_addr(st + SL::kGrad), T.grad + row0 * 128, gb, full);
+                bulk_load(smem_addr(st + SL::kM), T.m + row0 * 128, mb, full);
+                if (OPT == OPT_ADAM) bulk_load(smem_addr(st + SL::kV), T.v + row0 * 128, mb, full);
+                StageHeader h;
+                h.w = T.w; h.scale = T.scale; h.m = T.m; h.v = T.v;
+                h.row0 = row0; h.nrows = nrows; h.tensor_id = T.tensor_id; h.slot = T.slot;
+                h.s_old = 1.0f; h.s_new = 1.0f; h.inv_new = 1.0f;
+                if (MODE == MODE_TENSOR_AMAX) {
+                    h.s_old = load_scale(T.scale, 0, bf16_scale);
+                    if (local == 0) scratch_s_old[T.slot] = h.s_old;
+                }
+                if (MODE == MODE_TENSOR_APPLY) {
+                    h.s_old = scratch_s_old[T.slot];
+                    uint32_t bits;
+                    make_scale<FMT>(__uint_as_float(scratch_amax[T.slot]), bf16_scale, h.s_new, h.inv_new, bits);
+                    if (local == 0) {
+                        store_scale(T.scale, 0, bf16_scale, h.s_new, bits);
+                        scratch_amax_next[T.slot] = 0u;
+                    }
+                }
+                *reinterpret_cast<StageHeader*>(st + SL::kHeader) = h;
+            }
+            if (MODE == MODE_BLOCK && lane < static_cast<int>(nrows))
+                reinterpret_cast<float*>(st + SL::kScales)[lane] = load_scale(T.scale, row0 + lane, bf16_scale);
+            __syncwarp();
+            if (lane == 0) mbar_arrive(full);
+            ++issued;
+        }
+        if (!ok) {
+            // leave only after the copies already issued have landed (bounded)
+            const uint32_t pending = issued < static_cast<uint32_t>(S) ? issued : static_cast<uint32_t>(S);
+            for (uint32_t k = 0; k < pending; ++k) {
+                const uint32_t it = issued - 1 - k;
+                mbar_wait(full0 + 8 * (it % S), (it / S) & 1, status, 2u);
+            }
+        }
+        return;
+    }
+
+    // -------------------------------- consumers --------------------------------
+    const int r = warp * 4;                       // first of this warp's 4 rows in a unit
+    uint32_t cur_slot = 0xFFFFFFFFu;
+    float run_max = 0.0f;                         // MODE_TENSOR_AMAX
+    for (uint32_t it = 0; it < n_my; ++it) {
+        const uint32_t s = it % S, ph = (it / S) & 1;
+        if (!mbar_wait(full0 + 8 * s, ph, status, 3u)) return;
+        const uint8_t* st = stage0 + static_cast<size_t>(s) * SL::kBytes;
+        const StageHeader h = *reinterpret_cast<const StageHeader*>(st + SL::kHeader);
+
+        Lane4<OPT> L[4];
+        float amax[4];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            const int row = r + k;
+            const bool valid = row < static_cast<int>(h.nrows);
+            uint32_t codes = 0;
+            float g[4] = {0.f, 0.f, 0.f, 0.f}, m[4] = {0.f, 0.f, 0.f, 0.f}, v[4] = {0.f, 0.f, 0.f, 0.f}, vt[4];
+            float s_old = MODE == MODE_BLOCK ? 1.0f : h.s_old;
+            if (valid) {
+                if (FMT == FMT_FP8) codes = *reinterpret_cast<const uint32_t*>(st + SL::kCodes + row * 128 + lane * 4);
+                else codes = *reinterpret_cast<const uint16_t*>(st + SL::kCodes + row * 64 + lane * 2);
+                const uint2 gr = *reinterpret_cast<const uint2*>(st + SL::kGrad + row * 256 + lane * 8);
+                g[0] = __uint_as_float(gr.x << 16); g[1] = __uint_as_float(gr.x & 0xFFFF0000u);
+                g[2] = __uint_as_float(gr.y << 16); g[3] = __uint_as_float(gr.y & 0xFFFF0000u);
+                const float4 mr = *reinterpret_cast<const float4*>(st + SL::kM + row * 512 + lane * 16);
+                m[0] = mr.x; m[1] = mr.y; m[2] = mr.z; m[3] = mr.w;
+                if (OPT == OPT_ADAM) {
+                    const float4 vr = *reinterpret_cast<const float4*>(st + SL::kV + row * 512 + lane * 16);
+                    v[0] = vr.x; v[1] = vr.y; v[2] = vr.z; v[3] = vr.w;
+                }
+                if (MODE == MODE_BLOCK) s_old = reinterpret_cast<const float*>(st + SL::kScales)[row];
+            }
+            amax[k] = front4<FMT, OPT>(P, codes, g, m, v, s_old, valid ? 4 : 0, L[k], vt);
+            if (OPT == OPT_ADAM && MODE != MODE_TENSOR_AMAX && valid)
+                *reinterpret_cast<float4*>(h.v + (h.row0 + row) * 128 + lane * 4) = make_float4(vt[0], vt[1], vt[2], vt[3]);
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(empty0 + 8 * s);   // the stage may be refilled
+
+        if (MODE == MODE_TENSOR_AMAX) {
+            if (h.slot != cur_slot) {
+                if (cur_slot != 0xFFFFFFFFu) {
+                    float z = run_max;
+#pragma unroll
+                    for (int o = 16; o > 0; o >>= 1) z = fmaxf(z, __shfl_xor_sync(0xFFFFFFFFu, z, o));
+                    if (lane == 0) atomicMax(scratch_amax + cur_slot, __float_as_uint(z));
+                }
+                cur_slot = h.slot;
+                run_max = 0.0f;
+            }
+            run_max = fmaxf(fmaxf(run_max, fmaxf(amax[0], amax[1])), fmaxf(amax[2], amax[3]));
+            continue;
+        }
+
+        float s_k[4], inv_k[4];
+        if (MODE == MODE_BLOCK) {
+            const float my_amax = reduce_rows4s(amax, lane);      // row r + lane / 8
+            float s_mine, inv_mine;
+            uint32_t bits_mine;
+            make_scale<FMT>(my_amax, bf16_scale, s_mine, inv_mine, bits_mine);
+            const int g8 = lane >> 3;
+            if ((lane & 7) == 0 && r + g8 < static_cast<int>(h.nrows))
+                store_scale(h.scale, h.row0 + r + g8, bf16_scale, s_mine, bits_mine);
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                s_k[k] = __shfl_sync(0xFFFFFFFFu, s_mine, 8 * k);
+                inv_k[k] = __shfl_sync(0xFFFFFFFFu, inv_mine, 8 * k);
+            }
+        } else {
+#pragma unroll
+            for (int k = 0; k < 4; ++k) { s_k[k] = h.s_new; inv_k[k] = h.inv_new; }
+        }
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            const int row = r + k;
+            if (row >= static_cast<int>(h.nrows)) continue;
+            const uint64_t i0 = (h.row0 + row) * 128 + lane * 4;
+            uint32_t word[4] = {0u, 0u, 0u, 0u};
+            if (RND == RND_SR) {
+                const uint4 rw = philox4x32_10(static_cast<uint32_t>(i0 >> 2), h.tensor_id, P.step_lo, P.step_hi, P);
+                word[0] = rw.x; word[1] = rw.y; word[2] = rw.z; word[3] = rw.w;
+            }
+            float mh[4];
+            const uint32_t codes = back4<FMT, OPT, RND>(P, word, s_k[k], inv_k[k], L[k], mh);
+            if (FMT == FMT_FP8) *reinterpret_cast<uint32_t*>(h.w + i0) = codes;
+            else *reinterpret_cast<uint16_t*>(h.w + (i0 >> 1)) = static_cast<uint16_t>(codes);
+            *reinterpret_cast<float4*>(h.m + i0) = make_float4(mh[0], mh[1], mh[2], mh[3]);
+        }
+    }
+    if (MODE == MODE_TENSOR_AMAX && cur_slot != 0xFFFFFFFFu) {
+        float z = run_max;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) z = fmaxf(z, __shfl_xor_sync(0xFFFFFFFFu, z, o));
+        if (lane == 0) atomicMax(scratch_amax + cur_slot, __float_as_uint(z));
+    }
+}
+
+// ---------------------------------------------------------------------------
+template <int FMT, int OPT, int RND, int MODE>
+static cudaError_t launch_one(const TensorDesc* descs, const uint32_t* unit_tensor, uint32_t n_units, const StepParams& P,
+                              int bf16_scale, uint32_t* amax, uint32_t* amax_next, float* s_old, bool reverse,
+                              uint32_t* status, int grid_cap, cudaStream_t stream) {
+    using SL = StageLayout<FMT, OPT>;
+    static bool configured = false;
+    auto kernel = eco_stream_kernel<FMT, OPT, RND, MODE>;
+    if (!configured) {
+        cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SL::kSmem);
+        if (e != cudaSuccess) return e;
+        configured = true;
+    }
+    const uint32_t grid = n_units < static_cast<uint32_t>(grid_cap) ? n_units : static_cast<uint32_t>(grid_cap);
+    kernel<<<grid, kStreamThreads, SL::kSmem, stream>>>(descs, unit_tensor, n_units, P, bf16_scale, amax, amax_next,
+                                                        s_old, reverse ? 1 : 0, status);
+    return cudaGetLastError();
+}
+
+#define ECO_S_FMT(fmt, ...)                                            \
+    if ((fmt) == FMT_FP8) { constexpr int F = FMT_FP8; __VA_ARGS__ }   \
+    else { constexpr int F = FMT_INT4; __VA_ARGS__ }
+#define ECO_S_OPT(opt, ...)                                              \
+    if ((opt) == OPT_SGDM) { constexpr int O = OPT_SGDM; __VA_ARGS__ }   \
+    else { constexpr int O = OPT_ADAM; __VA_ARGS__ }
+#define ECO_S_RND(rnd, ...)                                            \
+    if ((rnd) == RND_RTN) { constexpr int R = RND_RTN; __VA_ARGS__ }   \
+    else { constexpr int R = RND_SR; __VA_ARGS__ }
+
+cudaError_t launch_stream(const LaunchConfig& c, int mode, const TensorDesc* descs, const uint32_t* unit_tensor,
+                          uint32_t n_units, const StepParams& P, uint32_t* amax, uint32_t* amax_next, float* s_old,
+                          bool reverse, uint32_t* status, int grid_cap, cudaStream_t stream) {
+    if (n_units == 0) return cudaSuccess;
+    if (mode == STREAM_TENSOR_AMAX) {
+        ECO_S_FMT(c.format, ECO_S_OPT(c.optimizer, {
+            return launch_one<F, O, RND_RTN, MODE_TENSOR_AMAX>(descs, unit_tensor, n_units, P, c.bf16_scale, amax,
+                                                               amax_next, s_old, reverse, status, grid_cap, stream);
+        }))
+    }
+    ECO_S_FMT(c.format, ECO_S_OPT(c.optimizer, ECO_S_RND(c.rounding, {
+        if (mode == STREAM_BLOCK)
+            return launch_one<F, O, R, MODE_BLOCK>(descs, unit_tensor, n_units, P, c.bf16_scale, amax, amax_next, s_old,
+                                                   reverse, status, grid_cap, stream);
+        return launch_one<F, O, R, MODE_TENSOR_APPLY>(descs, unit_tensor, n_units, P, c.bf16_scale, amax, amax_next,
+                                                      s_old, reverse, status, grid_cap, stream);
+    })))
+    return cudaErrorInvalidValue;
+}
+
+int stream_unit_rows() { return kUnitRows; }
+
+}  // namespace eco

@@ -24,7 +24,7 @@ ECO_OPT_SGDM, ECO_OPT_ADAM = 0, 1
 ECO_ROUND_NEAREST, ECO_ROUND_STOCHASTIC = 0, 1
 ECO_INJECT_NONE, ECO_INJECT_ECO = 0, 1
 
-EXPORTED = ("eco_create", "eco_step", "eco_step_host", "eco_destroy", "eco_last_error", "eco_quantize",
+EXPORTED = ("eco_create", "eco_step", "eco_step_host", "eco_check", "eco_destroy", "eco_last_error", "eco_quantize",
             "eco_set_option", "eco_num_launches", "eco_version")
 
 
@@ -67,6 +67,8 @@ def load_library() -> ctypes.CDLL:
         L.eco_step_host.argtypes = [ctypes.POINTER(eco_config), ctypes.POINTER(eco_tensor), ctypes.c_size_t,
                                     ctypes.c_int, f32, f32, f32, f32, u64, u64,
                                     ctypes.POINTER(u64), ctypes.POINTER(u64)]
+        L.eco_check.restype = ctypes.c_int
+        L.eco_check.argtypes = [vp, vp]
         L.eco_destroy.restype = ctypes.c_int
         L.eco_destroy.argtypes = [vp]
         L.eco_last_error.restype = ctypes.c_char_p
@@ -165,6 +167,13 @@ def eco_step_host(cfg: Config, tensors: Sequence[Tensor], lr: float, beta1: floa
     if st != ECO_OK:
         _raise(st)
     return up.value, down.value
+
+
+def eco_check(handle: int, stream: int = 0) -> None:
+    """Synchronize ``stream`` and raise if a bounded device-side wait expired.  See include/eco.h."""
+    st = load_library().eco_check(handle, stream)
+    if st != ECO_OK:
+        _raise(st, handle)
 
 
 def eco_destroy(handle: int) -> None:

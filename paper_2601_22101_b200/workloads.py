@@ -193,7 +193,26 @@ def shape_slice(w: Workload, max_rows: Optional[int] = None) -> Workload:
     return replace(w, name=w.name + "_slice", tensors=ts)
 
 
-BY_NAME = {"c1": c1, "c2": c2, "c3": c3, "c4": c4, "c5": c5}
+def c3_small() -> Workload:
+    """Two layers and a 32768-row embedding of the Gemma-3-1B-shaped set (profiling-sized: ~1 GB of state)."""
+    w = c3(layers=2, vocab=32768)
+    return replace(w, name=w.name + "_small")
+
+
+def c4_small() -> Workload:
+    """One layer (64 experts) of the sparse-MoE set (profiling-sized: ~1.5 GB of state)."""
+    w = c4(layers=1)
+    return replace(w, name=w.name + "_small")
+
+
+def c5_small() -> Workload:
+    """The dense layer and one MoE layer of 16 experts of the DeepSeek-MoE-shaped set (~1.4 GB of state)."""
+    w = c5(moe_layers=1, experts=16)
+    return replace(w, name=w.name + "_small")
+
+
+BY_NAME = {"c1": c1, "c2": c2, "c3": c3, "c4": c4, "c5": c5,
+           "c3s": c3_small, "c4s": c4_small, "c5s": c5_small}
 
 
 def _rng(w: Workload, t: TensorSpec, step: int, kind: int) -> np.random.Generator:
