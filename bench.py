@@ -40,13 +40,16 @@ def _workload(name: str):
 
 
 def _dominant_kernel(w) -> str:
+    """Name of the kernel that moves most of a step's bytes (full-size sets are made of whole 128-element rows,
+    which the persistent TMA-fed kernel takes)."""
     from paper_2601_22101_b200 import workloads as wl
     fmt = "fp8" if w.format == wl.FP8_E4M3 else "int4"
     opt = "adam" if w.optimizer == wl.ADAM else "sgdm"
     rnd = "sr" if w.rounding == wl.SR else "rtn"
-    kind = {wl.PER_BLOCK: "eco_block128_kernel", wl.PER_TENSOR: "eco_tensor_apply_kernel",
-            wl.PER_ROW: "eco_row_kernel"}[w.granularity]
-    return f"{kind}<{fmt},{opt},{rnd}>"
+    if w.granularity == wl.PER_ROW:
+        return f"eco_row_kernel<{fmt},{opt},{rnd}>"
+    mode = "block" if w.granularity == wl.PER_BLOCK else "tensor_apply"
+    return f"eco_stream_kernel<{fmt},{opt},{rnd},{mode}>"
 
 
 def _measured_peak():
