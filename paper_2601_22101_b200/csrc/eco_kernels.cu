@@ -241,9 +241,10 @@ __device__ __forceinline__ void quantize_lane(const float* x, uint8_t* w, uint64
     load_f32x4(x, i0, nvalid, vec, xv);
     uint32_t word[4] = {0u, 0u, 0u, 0u};
     if (RND == RND_SR) random_words4(P, tensor_id, i0, vec, word);
-    float q[4];
+    float y[4], q[4];
 #pragma unroll
-    for (int e = 0; e < 4; ++e) q[e] = round_to_grid<FMT, RND>(__fmul_rn(xv[e], s_inv), word[e]);
+    for (int e = 0; e < 4; ++e) y[e] = __fmul_rn(xv[e], s_inv);
+    round4<FMT, RND>(y, word, q);
     store_codes4<FMT>(w, i0, nvalid, vec, pack4<FMT>(q));
 }
 

@@ -94,22 +94,119 @@ __device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_
                  ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
 }
 
-__device__ __forceinline__ float reduce_rows4s(const float a[4], int lane) {
-    const bool b4 = lane & 16, b3 = lane & 8;
-    const float send_x = b4 ? a[0] : a[2], send_y = b4 ? a[1] : a[3];
-    const float keep_x = b4 ? a[2] : a[0], keep_y = b4 ? a[3] : a[1];
-    const float x = fmaxf(keep_x, __shfl_xor_sync(0xFFFFFFFFu, send_x, 16));
-    const float y = fmaxf(keep_y, __shfl_xor_sync(0xFFFFFFFFu, send_y, 16));
-    const float send = b3 ? x : y, keep = b3 ? y : x;
-    float z = fmaxf(keep, __shfl_xor_sync(0xFFFFFFFFu, send, 8));
-    z = fmaxf(z, __shfl_xor_sync(0xFFFFFFFFu, z, 4));
-    z = fmaxf(z, __shfl_xor_sync(0xFFFFFFFFu, z, 2));
-    z = fmaxf(z, __shfl_xor_sync(0xFFFFFFFFu, z, 1));
-    return z;
+// max |x| over the 32 lanes in one instruction (sm_100a warp reduction on binary32; NaN operands are
+// ignored, as by fmaxf).  Every lane receives the result.
+__device__ __forceinline__ float warp_amax(float x) {
+    float r;
+    asm volatile("redux.sync.max.abs.f32 %0, %1, 0xffffffff;" : "=f"(r) : "f"(x));
+    return r;
 }
 
 __device__ __forceinline__ uint32_t units_of(const TensorDesc& T) {
     return static_cast<uint32_t>((T.n_blocks + kUnitRows - 1) / kUnitRows);
+}
+
+// One unit (up to 32 rows of 128 elements) by the 8 consumer warps: warp w owns rows 4w..4w+3, lane l
+// elements 4l..4l+3 of each.  FULL: all 32 rows are present (every unit but the last of a tensor).
+template <int FMT, int OPT, int RND, int MODE, bool FULL>
+__device__ __forceinline__ void consume_unit(const StepParams& P, const int bf16_scale, const uint8_t* st,
+                                             const StageHeader* h, const uint32_t empty_bar, const int warp,
+                                             const int lane, uint32_t* scratch_amax, uint32_t& cur_slot,
+                                             float& run_max) {
+    using SL = StageLayout<FMT, OPT>;
+    const int r = warp * 4;
+    const int nrows = FULL ? kUnitRows : static_cast<int>(h->nrows);
+    const uint64_t i_first = (h->row0 + r) * 128 + lane * 4;      // element index of (row r, this lane)
+    float* const vp = h->v;
+
+    Lane4<OPT> L[4];
+    float amax[4];
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+        const int row = r + k;
+        const bool valid = FULL || row < nrows;
+        uint32_t codes = 0;
+        float g[4] = {0.f, 0.f, 0.f, 0.f}, m[4] = {0.f, 0.f, 0.f, 0.f}, v[4] = {0.f, 0.f, 0.f, 0.f}, vt[4];
+        float s_old = 1.0f;
+        if (valid) {
+            if (FMT == FMT_FP8) codes = *reinterpret_cast<const uint32_t*>(st + SL::kCodes + row * 128 + lane * 4);
+            else codes = *reinterpret_cast<const uint16_t*>(st + SL::kCodes + row * 64 + lane * 2);
+            const uint2 gr = *reinterpret_cast<const uint2*>(st + SL::kGrad + row * 256 + lane * 8);
+            g[0] = __uint_as_float(gr.x << 16); g[1] = __uint_as_float(gr.x & 0xFFFF0000u);
+            g[2] = __uint_as_float(gr.y << 16); g[3] = __uint_as_float(gr.y & 0xFFFF0000u);
+            const float4 mr = *reinterpret_cast<const float4*>(st + SL::kM + row * 512 + lane * 16);
+            m[0] = mr.x; m[1] = mr.y; m[2] = mr.z; m[3] = mr.w;
+            if (OPT == OPT_ADAM) {
+                const float4 vr = *reinterpret_cast<const float4*>(st + SL::kV + row * 512 + lane * 16);
+                v[0] = vr.x; v[1] = vr.y; v[2] = vr.z; v[3] = vr.w;
+            }
+            s_old = MODE == MODE_BLOCK ? reinterpret_cast<const float*>(st + SL::kScales)[row] : h->s_old;
+        }
+        amax[k] = front4<FMT, OPT>(P, codes, g, m, v, s_old, valid ? 4 : 0, L[k], vt);
+        if (OPT == OPT_ADAM && MODE != MODE_TENSOR_AMAX && valid)
+            *reinterpret_cast<float4*>(vp + i_first + k * 128) = make_float4(vt[0], vt[1], vt[2], vt[3]);
+    }
+    // everything needed later is read before the stage is handed back
+    uint8_t* const wp = h->w;
+    float* const mp = h->m;
+    void* const sp = h->scale;
+    const uint64_t row0 = h->row0;
+    const uint32_t tensor_id = h->tensor_id, slot = h->slot;
+    const float s_new = h->s_new, inv_new = h->inv_new;
+    __syncwarp();
+    if (lane == 0) mbar_arrive(empty_bar);          // the stage may be refilled
+
+    if (MODE == MODE_TENSOR_AMAX) {
+        if (slot != cur_slot) {
+            if (cur_slot != 0xFFFFFFFFu) {
+                const float z = warp_amax(run_max);
+                if (lane == 0) atomicMax(scratch_amax + cur_slot, __float_as_uint(z));
+            }
+            cur_slot = slot;
+            run_max = 0.0f;
+        }
+        run_max = fmaxf(fmaxf(run_max, fmaxf(amax[0], amax[1])), fmaxf(amax[2], amax[3]));
+        return;
+    }
+
+    float s_k[4], inv_k[4];
+    if (MODE == MODE_BLOCK) {
+        // row maxima: one warp reduction per row; lane group g = lane / 8 then derives the scale of row g
+        // and the four scales are broadcast from lanes 0, 8, 16, 24
+        float rmax[4];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) rmax[k] = warp_amax(amax[k]);
+        const int g8 = lane >> 3;
+        const float my_amax = g8 == 0 ? rmax[0] : (g8 == 1 ? rmax[1] : (g8 == 2 ? rmax[2] : rmax[3]));
+        float s_mine, inv_mine;
+        uint32_t bits_mine;
+        make_scale<FMT>(my_amax, bf16_scale, s_mine, inv_mine, bits_mine);
+        if ((lane & 7) == 0 && (FULL || r + g8 < nrows))
+            store_scale(sp, row0 + r + g8, bf16_scale, s_mine, bits_mine);
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            s_k[k] = __shfl_sync(0xFFFFFFFFu, s_mine, 8 * k);
+            inv_k[k] = __shfl_sync(0xFFFFFFFFu, inv_mine, 8 * k);
+        }
+    } else {
+#pragma unroll
+        for (int k = 0; k < 4; ++k) { s_k[k] = s_new; inv_k[k] = inv_new; }
+    }
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+        if (!FULL && r + k >= nrows) continue;
+        const uint64_t i0 = i_first + k * 128;
+        uint32_t word[4] = {0u, 0u, 0u, 0u};
+        if (RND == RND_SR) {
+            const uint4 rw = philox4x32_10(static_cast<uint32_t>(i0 >> 2), tensor_id, P.step_lo, P.step_hi, P);
+            word[0] = rw.x; word[1] = rw.y; word[2] = rw.z; word[3] = rw.w;
+        }
+        float mh[4];
+        const uint32_t codes = back4<FMT, OPT, RND>(P, word, s_k[k], inv_k[k], L[k], mh);
+        if (FMT == FMT_FP8) *reinterpret_cast<uint32_t*>(wp + i0) = codes;
+        else *reinterpret_cast<uint16_t*>(wp + (i0 >> 1)) = static_cast<uint16_t>(codes);
+        *reinterpret_cast<float4*>(mp + i0) = make_float4(mh[0], mh[1], mh[2], mh[3]);
+    }
 }
 
 // ---------------------------------------------------------------------------
@@ -210,99 +307,21 @@ eco_stream_kernel(const TensorDesc* __restrict__ descs, const uint32_t* __restri
     }
 
     // -------------------------------- consumers --------------------------------
-    const int r = warp * 4;                       // first of this warp's 4 rows in a unit
     uint32_t cur_slot = 0xFFFFFFFFu;
     float run_max = 0.0f;                         // MODE_TENSOR_AMAX
     for (uint32_t it = 0; it < n_my; ++it) {
         const uint32_t s = it % S, ph = (it / S) & 1;
         if (!mbar_wait(full0 + 8 * s, ph, status, 3u)) return;
         const uint8_t* st = stage0 + static_cast<size_t>(s) * SL::kBytes;
-        const StageHeader h = *reinterpret_cast<const StageHeader*>(st + SL::kHeader);
-
-        Lane4<OPT> L[4];
-        float amax[4];
-#pragma unroll
-        for (int k = 0; k < 4; ++k) {
-            const int row = r + k;
-            const bool valid = row < static_cast<int>(h.nrows);
-            uint32_t codes = 0;
-            float g[4] = {0.f, 0.f, 0.f, 0.f}, m[4] = {0.f, 0.f, 0.f, 0.f}, v[4] = {0.f, 0.f, 0.f, 0.f}, vt[4];
-            float s_old = MODE == MODE_BLOCK ? 1.0f : h.s_old;
-            if (valid) {
-                if (FMT == FMT_FP8) codes = *reinterpret_cast<const uint32_t*>(st + SL::kCodes + row * 128 + lane * 4);
-                else codes = *reinterpret_cast<const uint16_t*>(st + SL::kCodes + row * 64 + lane * 2);
-                const uint2 gr = *reinterpret_cast<const uint2*>(st + SL::kGrad + row * 256 + lane * 8);
-                g[0] = __uint_as_float(gr.x << 16); g[1] = __uint_as_float(gr.x & 0xFFFF0000u);
-                g[2] = __uint_as_float(gr.y << 16); g[3] = __uint_as_float(gr.y & 0xFFFF0000u);
-                const float4 mr = *reinterpret_cast<const float4*>(st + SL::kM + row * 512 + lane * 16);
-                m[0] = mr.x; m[1] = mr.y; m[2] = mr.z; m[3] = mr.w;
-                if (OPT == OPT_ADAM) {
-                    const float4 vr = *reinterpret_cast<const float4*>(st + SL::kV + row * 512 + lane * 16);
-                    v[0] = vr.x; v[1] = vr.y; v[2] = vr.z; v[3] = vr.w;
-                }
-                if (MODE == MODE_BLOCK) s_old = reinterpret_cast<const float*>(st + SL::kScales)[row];
-            }
-            amax[k] = front4<FMT, OPT>(P, codes, g, m, v, s_old, valid ? 4 : 0, L[k], vt);
-            if (OPT == OPT_ADAM && MODE != MODE_TENSOR_AMAX && valid)
-                *reinterpret_cast<float4*>(h.v + (h.row0 + row) * 128 + lane * 4) = make_float4(vt[0], vt[1], vt[2], vt[3]);
-        }
-        __syncwarp();
-        if (lane == 0) mbar_arrive(empty0 + 8 * s);   // the stage may be refilled
-
-        if (MODE == MODE_TENSOR_AMAX) {
-            if (h.slot != cur_slot) {
-                if (cur_slot != 0xFFFFFFFFu) {
-                    float z = run_max;
-#pragma unroll
-                    for (int o = 16; o > 0; o >>= 1) z = fmaxf(z, __shfl_xor_sync(0xFFFFFFFFu, z, o));
-                    if (lane == 0) atomicMax(scratch_amax + cur_slot, __float_as_uint(z));
-                }
-                cur_slot = h.slot;
-                run_max = 0.0f;
-            }
-            run_max = fmaxf(fmaxf(run_max, fmaxf(amax[0], amax[1])), fmaxf(amax[2], amax[3]));
-            continue;
-        }
-
-        float s_k[4], inv_k[4];
-        if (MODE == MODE_BLOCK) {
-            const float my_amax = reduce_rows4s(amax, lane);      // row r + lane / 8
-            float s_mine, inv_mine;
-            uint32_t bits_mine;
-            make_scale<FMT>(my_amax, bf16_scale, s_mine, inv_mine, bits_mine);
-            const int g8 = lane >> 3;
-            if ((lane & 7) == 0 && r + g8 < static_cast<int>(h.nrows))
-                store_scale(h.scale, h.row0 + r + g8, bf16_scale, s_mine, bits_mine);
-#pragma unroll
-            for (int k = 0; k < 4; ++k) {
-                s_k[k] = __shfl_sync(0xFFFFFFFFu, s_mine, 8 * k);
-                inv_k[k] = __shfl_sync(0xFFFFFFFFu, inv_mine, 8 * k);
-            }
-        } else {
-#pragma unroll
-            for (int k = 0; k < 4; ++k) { s_k[k] = h.s_new; inv_k[k] = h.inv_new; }
-        }
-#pragma unroll
-        for (int k = 0; k < 4; ++k) {
-            const int row = r + k;
-            if (row >= static_cast<int>(h.nrows)) continue;
-            const uint64_t i0 = (h.row0 + row) * 128 + lane * 4;
-            uint32_t word[4] = {0u, 0u, 0u, 0u};
-            if (RND == RND_SR) {
-                const uint4 rw = philox4x32_10(static_cast<uint32_t>(i0 >> 2), h.tensor_id, P.step_lo, P.step_hi, P);
-                word[0] = rw.x; word[1] = rw.y; word[2] = rw.z; word[3] = rw.w;
-            }
-            float mh[4];
-            const uint32_t codes = back4<FMT, OPT, RND>(P, word, s_k[k], inv_k[k], L[k], mh);
-            if (FMT == FMT_FP8) *reinterpret_cast<uint32_t*>(h.w + i0) = codes;
-            else *reinterpret_cast<uint16_t*>(h.w + (i0 >> 1)) = static_cast<uint16_t>(codes);
-            *reinterpret_cast<float4*>(h.m + i0) = make_float4(mh[0], mh[1], mh[2], mh[3]);
-        }
+        const StageHeader* h = reinterpret_cast<const StageHeader*>(st + SL::kHeader);
+        const uint32_t empty = empty0 + 8 * s;
+        if (h->nrows == kUnitRows)
+            consume_unit<FMT, OPT, RND, MODE, true>(P, bf16_scale, st, h, empty, warp, lane, scratch_amax, cur_slot, run_max);
+        else
+            consume_unit<FMT, OPT, RND, MODE, false>(P, bf16_scale, st, h, empty, warp, lane, scratch_amax, cur_slot, run_max);
     }
     if (MODE == MODE_TENSOR_AMAX && cur_slot != 0xFFFFFFFFu) {
-        float z = run_max;
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) z = fmaxf(z, __shfl_xor_sync(0xFFFFFFFFu, z, o));
+        const float z = warp_amax(run_max);
         if (lane == 0) atomicMax(scratch_amax + cur_slot, __float_as_uint(z));
     }
 }

@@ -211,6 +211,36 @@ def c5_small() -> Workload:
     return replace(w, name=w.name + "_small")
 
 
+def shard(w: Workload, rank: int, world: int) -> Workload:
+    """The tensors rank `rank` of `world` owns when a parameter set is split by whole tensors.
+
+    Tensors never interact in the step (a scale block lies inside one tensor) and the random stream is
+    keyed by (tensor_id, element index), so any split by whole tensors gives the same bits as the
+    unsplit set with no communication.  Assignment: largest tensor first, each to the rank with the
+    fewest parameters so far (ties to the lowest rank); deterministic, so every rank derives the same
+    partition without talking to the others."""
+    if not (0 <= rank < world):
+        raise ValueError("rank must be in [0, world)")
+    load = [0] * world
+    mine = []
+    order = sorted(range(len(w.tensors)), key=lambda i: (-w.tensors[i].numel, i))
+    for i in order:
+        r = min(range(world), key=lambda k: (load[k], k))
+        load[r] += w.tensors[i].numel
+        if r == rank:
+            mine.append(i)
+    mine.sort()
+    return replace(w, name=f"{w.name}_shard{rank}of{world}", tensors=[w.tensors[i] for i in mine])
+
+
+def replicate(w: Workload, copies: int) -> Workload:
+    """`copies` parameter sets of the shape of `w` as one job (weak scaling: the job grows with the number
+    of ranks); tensor ids stay unique so that every copy draws its own random stream."""
+    n = len(w.tensors)
+    ts = [replace(t, name=f"copy{c}.{t.name}", tensor_id=c * n + t.tensor_id) for c in range(copies) for t in w.tensors]
+    return replace(w, name=f"{w.name}_x{copies}", tensors=ts)
+
+
 BY_NAME = {"c1": c1, "c2": c2, "c3": c3, "c4": c4, "c5": c5,
            "c3s": c3_small, "c4s": c4_small, "c5s": c5_small}
 
