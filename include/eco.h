@@ -142,6 +142,42 @@ eco_status eco_step_host(const eco_config* cfg, const eco_tensor* tensors, size_
                          uint64_t* h2d_bytes, uint64_t* d2h_bytes);
 
 /*
+ * eco_step_static -- the step of eco_step for ECO_SCALE_PER_TENSOR, for callers that must not
+ * allocate device memory.  (The paper has no counterpart: this is a packaging of the same
+ * Algorithm 1 arithmetic, not another method.)
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits -- a process whose framework has
+ * already reserved the whole device for its own caching allocator, a latency-critical loop that
+ * cannot afford the device-wide synchronization an allocation implies, or a host that forbids
+ * allocation after start-up.  eco_create allocates its tables and reduction slots with cudaMalloc;
+ * this call needs no context and allocates nothing, on the device or through any library.  Its
+ * tables and reduction slots live in one fixed array (about 135 KB) inside the loaded library image,
+ * which every GPU that loads the library holds until the process exits.
+ *
+ *   cfg, tensors, n   as eco_create (tensors are device buffers the caller owns); granularity must be
+ *                     ECO_SCALE_PER_TENSOR.
+ *   lr .. seed        as eco_step.          cuda_stream   as eco_step.
+ * Limits: n <= ECO_STATIC_MAX_TENSORS and at most 2^27 parameters in the list (32768 work units of
+ * 4096 parameters, each tensor rounded up to whole units); beyond either the call returns
+ * ECO_ERR_INVALID_ARG, says so in eco_last_error(NULL), and launches nothing.
+ * Behaviour to know about:
+ *   - The first call on each device looks up the array's device address (with that device current).
+ *     Make that first call outside any stream capture.
+ *   - All calls share the one array, which still holds the previous call's tables: every call
+ *     rewrites what it uses and zeroes its reduction slots first.  Two calls whose GPU work overlaps
+ *     (different streams, or different host threads) race on it; serialize them.
+ *   - The call returns after cuda_stream has finished this step (it waits for the stream), unlike
+ *     eco_step.  Buffers are checked for NULL and alignment only, not for overlap or residency.
+ * Results are bit-identical to eco_create + eco_step on the same inputs.
+ * Errors: ECO_ERR_UNSUPPORTED (other granularity, unknown enum), ECO_ERR_INVALID_ARG,
+ * ECO_ERR_ALIGNMENT, ECO_ERR_CUDA.
+ */
+#define ECO_STATIC_MAX_TENSORS 64
+eco_status eco_step_static(const eco_config* cfg, const eco_tensor* tensors, size_t n, int device,
+                           float lr, float beta1, float beta2, float eps, uint64_t step, uint64_t seed,
+                           void* cuda_stream);
+
+/*
  * eco_check -- synchronize cuda_stream and report whether any kernel of this context gave up on a
  * device-side wait.  The streaming kernels wait on shared-memory barriers for their asynchronous
  * copies; every such wait is bounded (about two seconds of clock cycles), after which the kernel

@@ -6,6 +6,7 @@
 #include <cstdarg>
 #include <cstdio>
 #include <cstring>
+#include <mutex>
 #include <new>
 #include <string>
 #include <unordered_set>
@@ -583,6 +584,129 @@ eco_status eco_step_host(const eco_config* cfg, const eco_tensor* tensors, size_
     if (h2d_bytes) *h2d_bytes = up;
     if (d2h_bytes) *d2h_bytes = down;
     return bail(ECO_OK);
+}
+
+// ---------------------------------------------------------------------------
+// eco_step_static: the per-tensor-scale step with every byte of library-side
+// device memory taken from one fixed array that is part of the loaded module.
+// ---------------------------------------------------------------------------
+}  // extern "C"
+
+namespace {
+
+constexpr uint32_t kStaticMaxTensors = ECO_STATIC_MAX_TENSORS;
+constexpr uint32_t kStaticMaxUnits = 32768;   // work units of 4096 parameters: 2^27 parameters per call
+static_assert(sizeof(TensorDesc) % 8 == 0, "tables are laid out back to back");
+
+// Layout of the array: descriptors, amax slots of this step, amax slots the second kernel clears,
+// saved old scales, unit -> tensor table.
+struct StaticScratch {
+    TensorDesc descs[kStaticMaxTensors];
+    uint32_t amax[kStaticMaxTensors];
+    uint32_t amax_next[kStaticMaxTensors];
+    float s_old[kStaticMaxTensors];
+    uint32_t unit_tensor[kStaticMaxUnits];
+};
+
+// Lives in every GPU that loads the library, from load to exit (about 135 KB).  In host code this name
+// is only a handle: the device address comes from cudaGetSymbolAddress below.
+static __device__ __align__(256) unsigned char g_static_scratch[sizeof(StaticScratch)];
+
+constexpr int kMaxDevices = 64;
+std::mutex g_static_mutex;
+StaticScratch* g_static_ptr[kMaxDevices] = {};
+
+// Device address of the array on `device` (which must be current); resolved once per device.
+eco_status static_scratch_address(int device, StaticScratch** out) {
+    if (device < 0 || device >= kMaxDevices) return fail(nullptr, ECO_ERR_INVALID_ARG, "device ordinal %d out of range", device);
+    std::lock_guard<std::mutex> lock(g_static_mutex);
+    if (!g_static_ptr[device]) {
+        void* p = nullptr;
+        cudaError_t e = cudaGetSymbolAddress(&p, g_static_scratch);
+        if (e != cudaSuccess || !p)
+            return fail(nullptr, ECO_ERR_CUDA, "cudaGetSymbolAddress(static scratch) on device %d failed: %s", device,
+                        cudaGetErrorString(e));
+        g_static_ptr[device] = static_cast<StaticScratch*>(p);
+    }
+    *out = g_static_ptr[device];
+    return ECO_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+eco_status eco_step_static(const eco_config* cfg, const eco_tensor* tensors, size_t n, int device,
+                           float lr, float beta1, float beta2, float eps, uint64_t step, uint64_t seed,
+                           void* cuda_stream) {
+    if (eco_status st = check_config(cfg, true)) return st;
+    if (cfg->granularity != ECO_SCALE_PER_TENSOR)
+        return fail(nullptr, ECO_ERR_UNSUPPORTED, "eco_step_static handles ECO_SCALE_PER_TENSOR only");
+    if (!tensors || n == 0) return fail(nullptr, ECO_ERR_INVALID_ARG, "empty tensor list");
+    if (n > kStaticMaxTensors)
+        return fail(nullptr, ECO_ERR_INVALID_ARG, "eco_step_static takes at most %u tensors per call (got %zu)",
+                    kStaticMaxTensors, n);
+    if (eco_status st = check_hyper(nullptr, *cfg, lr, beta1, beta2, eps, step)) return st;
+    const bool adam = cfg->optimizer == ECO_OPT_ADAM;
+    const uint64_t rpu = static_cast<uint64_t>(eco::rows_per_unit());
+    static thread_local StaticScratch host;          // host image of the tables (no heap use either)
+    uint64_t units = 0, total = 0;
+    for (size_t i = 0; i < n; ++i) {
+        const eco_tensor& t = tensors[i];
+        if (eco_status st = check_shape(*cfg, t.rows, t.cols, i)) return st;
+        if (t.reserved != 0) return fail(nullptr, ECO_ERR_INVALID_ARG, "tensor %zu: reserved must be 0", i);
+        if (adam != (t.v != nullptr)) return fail(nullptr, ECO_ERR_INVALID_ARG, "tensor %zu: v must be given for Adam and NULL for SGDM", i);
+        for (size_t j = 0; j < i; ++j)
+            if (tensors[j].tensor_id == t.tensor_id) return fail(nullptr, ECO_ERR_INVALID_ARG, "tensor %zu: duplicate tensor_id %u", i, t.tensor_id);
+        const void* bufs[5] = {t.w, t.scale, t.grad, t.m, t.v};
+        const char* names[5] = {"w", "scale", "grad", "m", "v"};
+        for (int b = 0; b < (adam ? 5 : 4); ++b) {
+            if (!bufs[b]) return fail(nullptr, ECO_ERR_INVALID_ARG, "tensor %zu: %s is NULL", i, names[b]);
+            if (reinterpret_cast<uintptr_t>(bufs[b]) & 15) return fail(nullptr, ECO_ERR_ALIGNMENT, "tensor %zu: %s is not 16-byte aligned", i, names[b]);
+        }
+        TensorDesc d;
+        std::memset(&d, 0, sizeof d);
+        d.w = static_cast<uint8_t*>(t.w);
+        d.scale = t.scale;
+        d.grad = static_cast<const uint16_t*>(t.grad);
+        d.m = t.m;
+        d.v = t.v;
+        d.numel = static_cast<uint64_t>(t.rows) * static_cast<uint64_t>(t.cols);
+        d.cols = static_cast<uint32_t>(t.cols);
+        d.blocks_per_row = static_cast<uint32_t>((t.cols + 127) / 128);
+        d.n_blocks = (d.numel + 127) / 128;
+        d.tensor_id = t.tensor_id;
+        d.slot = static_cast<uint32_t>(i);
+        const uint64_t nu = (d.n_blocks + rpu - 1) / rpu;
+        total += d.numel;
+        if (units + nu > kStaticMaxUnits)
+            return fail(nullptr, ECO_ERR_INVALID_ARG,
+                        "eco_step_static takes at most %llu parameters per call (%u units of %llu); the list has more",
+                        static_cast<unsigned long long>(kStaticMaxUnits * rpu * 128), kStaticMaxUnits,
+                        static_cast<unsigned long long>(rpu * 128));
+        d.first_unit = static_cast<uint32_t>(units);
+        host.descs[i] = d;
+        for (uint64_t u = 0; u < nu; ++u) host.unit_tensor[units + u] = static_cast<uint32_t>(i);
+        units += nu;
+    }
+    (void)total;
+    ECO_CUDA(nullptr, cudaSetDevice(device));
+    StaticScratch* dev = nullptr;
+    if (eco_status st = static_scratch_address(device, &dev)) return st;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    // The array keeps whatever the previous call left: upload this call's tables and zero both amax ranges.
+    ECO_CUDA(nullptr, cudaMemcpyAsync(dev->descs, host.descs, n * sizeof(TensorDesc), cudaMemcpyHostToDevice, stream));
+    ECO_CUDA(nullptr, cudaMemcpyAsync(dev->unit_tensor, host.unit_tensor, units * sizeof(uint32_t), cudaMemcpyHostToDevice, stream));
+    ECO_CUDA(nullptr, cudaMemsetAsync(dev->amax, 0, 2 * kStaticMaxTensors * sizeof(uint32_t), stream));
+    const LaunchConfig lc = launch_config(*cfg);
+    const StepParams P = derive_params(*cfg, lr, beta1, beta2, eps, step, seed);
+    ECO_CUDA(nullptr, eco::launch_tensor_amax(lc, dev->descs, dev->unit_tensor, static_cast<uint32_t>(units), P, dev->amax,
+                                              dev->s_old, stream));
+    ECO_CUDA(nullptr, eco::launch_tensor_apply(lc, dev->descs, dev->unit_tensor, static_cast<uint32_t>(units), P, dev->amax,
+                                               dev->amax_next, dev->s_old, false, stream));
+    // the host image is reused by the next call on this thread: wait until the copies have read it
+    ECO_CUDA(nullptr, cudaStreamSynchronize(stream));
+    return ECO_OK;
 }
 
 }  // extern "C"

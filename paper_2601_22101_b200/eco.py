@@ -24,7 +24,7 @@ ECO_OPT_SGDM, ECO_OPT_ADAM = 0, 1
 ECO_ROUND_NEAREST, ECO_ROUND_STOCHASTIC = 0, 1
 ECO_INJECT_NONE, ECO_INJECT_ECO = 0, 1
 
-EXPORTED = ("eco_create", "eco_step", "eco_step_host", "eco_check", "eco_destroy", "eco_last_error", "eco_quantize",
+EXPORTED = ("eco_create", "eco_step", "eco_step_host", "eco_step_static", "eco_check", "eco_destroy", "eco_last_error", "eco_quantize",
             "eco_set_option", "eco_num_launches", "eco_version")
 
 
@@ -67,6 +67,9 @@ def load_library() -> ctypes.CDLL:
         L.eco_step_host.argtypes = [ctypes.POINTER(eco_config), ctypes.POINTER(eco_tensor), ctypes.c_size_t,
                                     ctypes.c_int, f32, f32, f32, f32, u64, u64,
                                     ctypes.POINTER(u64), ctypes.POINTER(u64)]
+        L.eco_step_static.restype = ctypes.c_int
+        L.eco_step_static.argtypes = [ctypes.POINTER(eco_config), ctypes.POINTER(eco_tensor), ctypes.c_size_t,
+                                      ctypes.c_int, f32, f32, f32, f32, u64, u64, vp]
         L.eco_check.restype = ctypes.c_int
         L.eco_check.argtypes = [vp, vp]
         L.eco_destroy.restype = ctypes.c_int
@@ -167,6 +170,19 @@ def eco_step_host(cfg: Config, tensors: Sequence[Tensor], lr: float, beta1: floa
     if st != ECO_OK:
         _raise(st)
     return up.value, down.value
+
+
+def eco_step_static(cfg: Config, tensors: Sequence[Tensor], lr: float, beta1: float, beta2: float, eps: float,
+                    step: int, seed: int, device: int = 0, stream: int = 0) -> None:
+    """One per-tensor-scale step with no context and no device allocation (the library's tables live in
+    a fixed array inside the loaded image).  For callers that cannot call cudaMalloc; see
+    ``eco_step_static`` in include/eco.h for the limits and the sharing rules."""
+    c = cfg.c()
+    arr = _tensor_array(tensors)
+    st = load_library().eco_step_static(ctypes.byref(c), arr, len(tensors), device, lr, beta1, beta2, eps,
+                                        step, seed, stream)
+    if st != ECO_OK:
+        _raise(st)
 
 
 def eco_check(handle: int, stream: int = 0) -> None:
