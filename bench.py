@@ -222,8 +222,8 @@ def run_e2e(w, device: int, steps: int, max_host_gb: float):
     torch.cuda.synchronize(device)
     el = time.perf_counter() - t0
     return {"value": ws.numel * steps / el, "unit": UNIT, "h2d_bytes_per_step": up, "d2h_bytes_per_step": down,
-            "steps": steps, "params_per_step": ws.numel,
-            "sample": f"first {len(picked)} of {len(w.tensors)} tensors held in pinned host memory"}
+            "steps": steps, "params_per_step": ws.numel, "seconds": el,
+            "sample": f"first {len(picked)} of {len(w.tensors)} tensors per GPU held in pinned host memory"}
 
 
 def main():
@@ -233,6 +233,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--workload", default="c4", choices=["c1", "c2", "c3", "c4", "c5", "c3s", "c4s", "c5s"])
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--also", default="c3,c5", help="comma-separated workloads timed after the headline one and "
+                    "reported under other_workloads (device-resident timing only)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--e2e-steps", type=int, default=2)
@@ -264,12 +266,60 @@ def main():
         k, v = o.split("=")
         eco.eco_set_option(k, int(v))
 
-    w = _workload(args.workload)
-    st = DeviceState(w, local)
-    st.init_on_device(seed=1234 + rank)
-    st.set_grads_on_device(seed=4321 + rank)
-    st.create()
-    launches_per_step = eco.eco_num_launches(st.handle)
+    def time_workload(w_global, steps, warmup, sample_clocks):
+        """Device-resident timing of `steps` eco_steps of this rank's shard; returns a dict (rank 0) or None."""
+        w_rank = wl.shard(wl.replicate(w_global, world), rank, world) if world > 1 else w_global
+        st = DeviceState(w_rank, local)
+        st.init_on_device(seed=1234 + rank)
+        st.set_grads_on_device(seed=4321 + rank)
+        st.create()
+        launches_per_step = eco.eco_num_launches(st.handle)
+        step_no = 0
+        for _ in range(max(warmup, 3)):
+            step_no += 1
+            st.step(step_no, stream.cuda_stream)
+        barrier()
+        sampler = ClockSampler(local) if sample_clocks else None
+        if sampler:
+            sampler.start()
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        ev0.record(stream)
+        for _ in range(steps):
+            step_no += 1
+            st.step(step_no, stream.cuda_stream)
+        ev1.record(stream)
+        barrier()
+        clocks = sampler.stop() if sampler else None
+        eco.eco_check(st.handle, stream.cuda_stream)
+        ms = ev0.elapsed_time(ev1)
+        if world > 1:
+            t = torch.tensor([ms], device="cuda", dtype=torch.float64)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms = float(t.item())
+        ms_per_step = ms / steps
+        state_bytes = st.device_bytes()
+        st.destroy()
+        del st
+        torch.cuda.empty_cache()
+        if rank != 0:
+            return None
+        peak, peak_src = _measured_peak()
+        bpp = w_global.algorithmic_bytes_per_param()
+        params_per_rank = w_rank.numel
+        achieved = params_per_rank * bpp / (ms_per_step * 1e-3) / 1e9
+        kern = _dominant_kernel(w_global)
+        tr = NCU_DRAM_BYTES_PER_PARAM.get(kern)
+        return {
+            "workload": w_global.name, "params_per_gpu": params_per_rank, "tensors_per_gpu": len(w_rank.tensors),
+            "ms_per_step": ms_per_step, "value": params_per_rank * world / (ms_per_step * 1e-3),
+            "launches_per_step": launches_per_step, "state_bytes_on_device": state_bytes, "clocks": clocks,
+            "roofline": {"bound": "hbm", "kernel": kern, "achieved": achieved, "peak": peak, "unit": "GB/s",
+                         "frac": achieved / peak, "peak_source": peak_src,
+                         "frac_of_nominal_8000": achieved / 8000.0,
+                         "algorithmic_bytes_per_param": bpp,
+                         "traffic": (tr * params_per_rank if tr else None)},
+        }
+
     stream = torch.cuda.current_stream()
 
     def barrier():
@@ -278,57 +328,42 @@ def main():
             dist.barrier()
         torch.cuda.synchronize()
 
-    step_no = 0
-    for _ in range(max(args.warmup, 3)):
-        step_no += 1
-        st.step(step_no, stream.cuda_stream)
-    barrier()
-    sampler = ClockSampler(local)
-    sampler.start()
-    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    ev0.record(stream)
-    for _ in range(args.steps):
-        step_no += 1
-        st.step(step_no, stream.cuda_stream)
-    ev1.record(stream)
-    barrier()
-    clocks = sampler.stop()
-    ms = ev0.elapsed_time(ev1)
-    if world > 1:
-        t = torch.tensor([ms], device="cuda", dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
-    ms_per_step = ms / args.steps
-    value = w.numel * world / (ms_per_step * 1e-3)
+    w = _workload(args.workload)
+    head = time_workload(w, args.steps, args.warmup, True)
+    others = []
+    for name in [n for n in args.also.split(",") if n and n != args.workload]:
+        r = time_workload(_workload(name), min(args.steps, 20), 3, True)
+        if r is not None:
+            others.append({k: r[k] for k in ("workload", "params_per_gpu", "ms_per_step", "value", "launches_per_step",
+                                             "clocks", "roofline")})
 
     if rank == 0:
-        peak, peak_src = _measured_peak()
-        bpp = w.algorithmic_bytes_per_param()
-        achieved = w.numel * bpp / (ms_per_step * 1e-3) / 1e9
-        kern = _dominant_kernel(w)
-        tr = NCU_DRAM_BYTES_PER_PARAM.get(kern)
         out = {
-            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-            "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
+            "metric": METRIC, "value": head["value"], "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": max(args.warmup, 3), "ms_per_step": head["ms_per_step"], "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-            "config": {"workload": w.name, "params": w.numel, "tensors": len(w.tensors),
-                       "state_bytes_on_device": st.device_bytes(),
+            "config": {"workload": w.name, "params_per_gpu": head["params_per_gpu"],
+                       "tensors_per_gpu": head["tensors_per_gpu"],
+                       "state_bytes_on_device": head["state_bytes_on_device"],
                        "l2": "inputs much larger than the 126 MB L2, streamed once per step (no flush needed)",
-                       "replicas": world},
-            "gpu_launches": launches_per_step * args.steps,
-            "clocks": clocks,
-            "roofline": {"bound": "hbm", "kernel": kern, "achieved": achieved, "peak": peak, "unit": "GB/s",
-                         "frac": achieved / peak, "peak_source": peak_src,
-                         "frac_of_nominal_8000": achieved / 8000.0,
-                         "algorithmic_bytes_per_param": bpp,
-                         "traffic": (tr * w.numel if tr else None)},
+                       "sharding": "whole tensors per rank, no data-path collective" if world > 1 else "single GPU"},
+            "gpu_launches": head["launches_per_step"] * args.steps,
+            "clocks": head["clocks"],
+            "roofline": head["roofline"],
+            "other_workloads": others,
         }
-    st.destroy()
+    if not args.no_e2e:
+        # every rank steps its own host-resident shard; the job's time is the slowest rank's
+        barrier()
+        e2e = run_e2e(w, local, args.e2e_steps, args.e2e_host_gb)
+        if world > 1:
+            t = torch.tensor([e2e["seconds"]], device="cuda", dtype=torch.float64)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            e2e["seconds"] = float(t.item())
+            e2e["value"] = e2e["params_per_step"] * world * e2e["steps"] / e2e["seconds"]
+        if rank == 0:
+            out["e2e"] = e2e
     if rank == 0:
-        if not args.no_e2e:
-            del st
-            torch.cuda.empty_cache()
-            out["e2e"] = run_e2e(w, local, args.e2e_steps, args.e2e_host_gb)
         if not args.no_cpu_baseline and world == 1:
             out["cpu_baseline"], _, _ = cpu_baseline(w)
         print(json.dumps(out))
