@@ -53,6 +53,7 @@ struct eco_ctx {
     uint32_t* d_amax[2] = {nullptr, nullptr};
     float* d_s_old = nullptr;
     uint32_t* d_status = nullptr;
+    uint32_t* d_tickets = nullptr;
     int grid_cap = 296;
     uint64_t calls = 0;
     bool reverse_pass2 = true;
@@ -394,6 +395,8 @@ eco_status eco_create(eco_ctx** out, const eco_config* cfg, const eco_tensor* te
     }
     ECO_CUDA_CTX(cudaMalloc(&ctx->d_status, sizeof(uint32_t)));
     ECO_CUDA_CTX(cudaMemset(ctx->d_status, 0, sizeof(uint32_t)));
+    ECO_CUDA_CTX(cudaMalloc(&ctx->d_tickets, 2 * sizeof(uint32_t)));
+    ECO_CUDA_CTX(cudaMemset(ctx->d_tickets, 0, 2 * sizeof(uint32_t)));
     ECO_CUDA_CTX(cudaDeviceSynchronize());
 #undef ECO_CUDA_CTX
     *out = ctx;
@@ -413,18 +416,18 @@ eco_status eco_step(eco_ctx* ctx, float lr, float beta1, float beta2, float eps,
         switch (L.kind) {
             case KIND_BLOCK_FAST:
                 ECO_CUDA(ctx, eco::launch_stream(ctx->lc, eco::STREAM_BLOCK, descs, units, L.n_units, P, nullptr, nullptr,
-                                                 nullptr, false, ctx->d_status, ctx->grid_cap, stream));
+                                                 nullptr, false, ctx->d_tickets, ctx->d_status, ctx->grid_cap, stream));
                 break;
             case KIND_BLOCK_GENERIC:
                 ECO_CUDA(ctx, eco::launch_block128(ctx->lc, descs, units, L.n_units, true, P, stream));
                 break;
             case KIND_TENSOR_STREAM:
                 ECO_CUDA(ctx, eco::launch_stream(ctx->lc, eco::STREAM_TENSOR_AMAX, descs, units, L.n_units, P,
-                                                 ctx->d_amax[parity], nullptr, ctx->d_s_old, false, ctx->d_status,
+                                                 ctx->d_amax[parity], nullptr, ctx->d_s_old, false, ctx->d_tickets, ctx->d_status,
                                                  ctx->grid_cap, stream));
                 ECO_CUDA(ctx, eco::launch_stream(ctx->lc, eco::STREAM_TENSOR_APPLY, descs, units, L.n_units, P,
                                                  ctx->d_amax[parity], ctx->d_amax[parity ^ 1], ctx->d_s_old,
-                                                 ctx->reverse_pass2, ctx->d_status, ctx->grid_cap, stream));
+                                                 ctx->reverse_pass2, ctx->d_tickets, ctx->d_status, ctx->grid_cap, stream));
                 break;
             case KIND_ROW:
                 ECO_CUDA(ctx, eco::launch_row(ctx->lc, descs, units, L.n_units, P, stream));
@@ -461,6 +464,7 @@ eco_status eco_destroy(eco_ctx* ctx) {
     cudaFree(ctx->d_amax[1]);
     cudaFree(ctx->d_s_old);
     cudaFree(ctx->d_status);
+    cudaFree(ctx->d_tickets);
     delete ctx;
     return ECO_OK;
 }

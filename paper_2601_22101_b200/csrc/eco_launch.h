@@ -24,11 +24,13 @@ int stream_unit_rows();
 enum : int { STREAM_BLOCK = 0, STREAM_TENSOR_AMAX = 1, STREAM_TENSOR_APPLY = 2 };
 enum : int { MODE_BLOCK = STREAM_BLOCK, MODE_TENSOR_AMAX = STREAM_TENSOR_AMAX, MODE_TENSOR_APPLY = STREAM_TENSOR_APPLY };
 
-// Persistent launch over n_units work units; grid = min(n_units, grid_cap).  `status` is a device word
-// that receives a non-zero code if a bounded wait inside the kernel expires.
+// Persistent launch over n_units work units; grid = min(n_units, grid_cap).  `tickets` are two device
+// words, zero before the first launch, that the kernel uses to hand out units and rewinds before it ends
+// (launches sharing them must be ordered on the device).  `status` is a device word that receives a
+// non-zero code if a bounded wait inside the kernel expires.
 cudaError_t launch_stream(const LaunchConfig& c, int mode, const TensorDesc* descs, const uint32_t* unit_tensor,
                           uint32_t n_units, const StepParams& P, uint32_t* amax, uint32_t* amax_next, float* s_old,
-                          bool reverse, uint32_t* status, int grid_cap, cudaStream_t stream);
+                          bool reverse, uint32_t* tickets, uint32_t* status, int grid_cap, cudaStream_t stream);
 
 cudaError_t launch_block128(const LaunchConfig& c, const TensorDesc* descs, const uint32_t* unit_tensor,
                             uint32_t n_units, bool generic, const StepParams& P, cudaStream_t stream);

@@ -26,6 +26,7 @@ constexpr int kConsumerWarps = 8;
 constexpr int kStreamThreads = (kConsumerWarps + 1) * 32;
 constexpr int kUnitRows = kConsumerWarps * 4;      // rows of 128 elements per unit
 constexpr long long kWaitLimitCycles = 4000000000LL;
+constexpr int kInterleave = 8;                     // regions of a block-scale launch walked concurrently
 
 // What the producer tells the consumers about a unit.
 struct StageHeader {
@@ -121,30 +122,44 @@ __device__ __forceinline__ void consume_unit(const StepParams& P, const int bf16
 
     Lane4<OPT> L[4];
     float amax[4];
+    {
+        float th[4][4], g[4][4], m[4][4], v[4][4], vt[4][4];
 #pragma unroll
-    for (int k = 0; k < 4; ++k) {
-        const int row = r + k;
-        const bool valid = FULL || row < nrows;
-        uint32_t codes = 0;
-        float g[4] = {0.f, 0.f, 0.f, 0.f}, m[4] = {0.f, 0.f, 0.f, 0.f}, v[4] = {0.f, 0.f, 0.f, 0.f}, vt[4];
-        float s_old = 1.0f;
-        if (valid) {
-            if (FMT == FMT_FP8) codes = *reinterpret_cast<const uint32_t*>(st + SL::kCodes + row * 128 + lane * 4);
-            else codes = *reinterpret_cast<const uint16_t*>(st + SL::kCodes + row * 64 + lane * 2);
-            const uint2 gr = *reinterpret_cast<const uint2*>(st + SL::kGrad + row * 256 + lane * 8);
-            g[0] = __uint_as_float(gr.x << 16); g[1] = __uint_as_float(gr.x & 0xFFFF0000u);
-            g[2] = __uint_as_float(gr.y << 16); g[3] = __uint_as_float(gr.y & 0xFFFF0000u);
-            const float4 mr = *reinterpret_cast<const float4*>(st + SL::kM + row * 512 + lane * 16);
-            m[0] = mr.x; m[1] = mr.y; m[2] = mr.z; m[3] = mr.w;
-            if (OPT == OPT_ADAM) {
-                const float4 vr = *reinterpret_cast<const float4*>(st + SL::kV + row * 512 + lane * 16);
-                v[0] = vr.x; v[1] = vr.y; v[2] = vr.z; v[3] = vr.w;
+        for (int k = 0; k < 4; ++k) {
+            const int row = r + k;
+            const bool valid = FULL || row < nrows;
+            uint32_t codes = 0;
+            float s_old = 1.0f;
+#pragma unroll
+            for (int e = 0; e < 4; ++e) { g[k][e] = 0.f; m[k][e] = 0.f; v[k][e] = 0.f; }
+            if (valid) {
+                if (FMT == FMT_FP8) codes = *reinterpret_cast<const uint32_t*>(st + SL::kCodes + row * 128 + lane * 4);
+                else codes = *reinterpret_cast<const uint16_t*>(st + SL::kCodes + row * 64 + lane * 2);
+                const uint2 gr = *reinterpret_cast<const uint2*>(st + SL::kGrad + row * 256 + lane * 8);
+                g[k][0] = __uint_as_float(gr.x << 16); g[k][1] = __uint_as_float(gr.x & 0xFFFF0000u);
+                g[k][2] = __uint_as_float(gr.y << 16); g[k][3] = __uint_as_float(gr.y & 0xFFFF0000u);
+                const float4 mr = *reinterpret_cast<const float4*>(st + SL::kM + row * 512 + lane * 16);
+                m[k][0] = mr.x; m[k][1] = mr.y; m[k][2] = mr.z; m[k][3] = mr.w;
+                if (OPT == OPT_ADAM) {
+                    const float4 vr = *reinterpret_cast<const float4*>(st + SL::kV + row * 512 + lane * 16);
+                    v[k][0] = vr.x; v[k][1] = vr.y; v[k][2] = vr.z; v[k][3] = vr.w;
+                }
+                s_old = MODE == MODE_BLOCK ? reinterpret_cast<const float*>(st + SL::kScales)[row] : h->s_old;
             }
-            s_old = MODE == MODE_BLOCK ? reinterpret_cast<const float*>(st + SL::kScales)[row] : h->s_old;
+            float val[4];
+            unpack4<FMT>(codes, val);
+#pragma unroll
+            for (int e = 0; e < 4; ++e) th[k][e] = __fmul_rn(val[e], s_old);
         }
-        amax[k] = front4<FMT, OPT>(P, codes, g, m, v, s_old, valid ? 4 : 0, L[k], vt);
-        if (OPT == OPT_ADAM && MODE != MODE_TENSOR_AMAX && valid)
-            *reinterpret_cast<float4*>(vp + i_first + k * 128) = make_float4(vt[0], vt[1], vt[2], vt[3]);
+        optim_rows<OPT, 4>(P, th, g, m, v, L, vt);
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            const bool valid = FULL || r + k < nrows;
+            amax[k] = 0.0f;
+            if (valid) amax[k] = fmaxf(fmaxf(fabsf(L[k].tht[0]), fabsf(L[k].tht[1])), fmaxf(fabsf(L[k].tht[2]), fabsf(L[k].tht[3])));
+            if (OPT == OPT_ADAM && MODE != MODE_TENSOR_AMAX && valid)
+                *reinterpret_cast<float4*>(vp + i_first + k * 128) = make_float4(vt[k][0], vt[k][1], vt[k][2], vt[k][3]);
+        }
     }
     // everything needed later is read before the stage is handed back
     uint8_t* const wp = h->w;
@@ -221,7 +236,8 @@ __global__ void __launch_bounds__(kStreamThreads, 2)
 eco_stream_kernel(const TensorDesc* __restrict__ descs, const uint32_t* __restrict__ unit_tensor,
                   const uint32_t n_units, const StepParams P, const int bf16_scale,
                   uint32_t* __restrict__ scratch_amax, uint32_t* __restrict__ scratch_amax_next,
-                  float* __restrict__ scratch_s_old, const int reverse, uint32_t* __restrict__ status) {
+                  float* __restrict__ scratch_s_old, const int reverse, const int interleave,
+                  uint32_t* __restrict__ tickets, uint32_t* __restrict__ status) {
     using SL = StageLayout<FMT, OPT>;
     constexpr int S = SL::kStages;
     extern __shared__ __align__(128) uint8_t smem[];
@@ -239,21 +255,31 @@ eco_stream_kernel(const TensorDesc* __restrict__ descs, const uint32_t* __restri
     }
     __syncthreads();
 
-    const uint32_t lo = static_cast<uint32_t>(static_cast<uint64_t>(n_units) * blockIdx.x / gridDim.x);
-    const uint32_t hi = static_cast<uint32_t>(static_cast<uint64_t>(n_units) * (blockIdx.x + 1) / gridDim.x);
-    const uint32_t n_my = hi - lo;
-    if (n_my == 0) return;
-
     if (warp == kConsumerWarps) {
         // ------------------------------ producer ------------------------------
-        uint32_t t = __ldg(unit_tensor + (reverse ? hi - 1 : lo));
-        TensorDesc T = descs[t];
-        uint32_t issued = 0;
+        // Units are handed out by a device-wide ticket counter, so CTAs that draw cheap units (tensors whose
+        // gradient is all zero skip the square roots and divisions) simply draw more of them.  Ticket t maps to
+        // unit (t mod W) * ceil(n / W) + t / W: W regions of the parameter set are walked at the same time, which
+        // mixes compute-heavy and memory-heavy tensors on every SM.  tickets[0] counts tickets, tickets[1] CTAs
+        // that are done drawing; the last one rewinds both for the next launch.
+        const uint32_t W = static_cast<uint32_t>(interleave);
+        const uint32_t per_region = (n_units + W - 1) / W;
+        const uint32_t n_tickets = per_region * W;
+        auto draw = [&]() -> uint32_t {
+            uint32_t t = 0;
+            if (lane == 0) t = atomicAdd(tickets, 1u);
+            return __shfl_sync(0xFFFFFFFFu, t, 0);
+        };
+        uint32_t ticket = draw();
+        uint32_t it = 0;
         bool ok = true;
-        for (uint32_t it = 0; it < n_my && ok; ++it) {
-            const uint32_t unit = reverse ? (hi - 1 - it) : (lo + it);
-            if (!reverse) { while (unit >= T.first_unit + units_of(T)) T = descs[++t]; }
-            else          { while (unit < T.first_unit) T = descs[--t]; }
+        while (ticket < n_tickets) {
+            const uint32_t next_ticket = draw();          // in flight while this unit is set up
+            const uint32_t cand = (ticket % W) * per_region + ticket / W;
+            ticket = next_ticket;
+            if (cand >= n_units) continue;
+            const uint32_t unit = reverse ? (n_units - 1 - cand) : cand;
+            const TensorDesc T = descs[__ldg(unit_tensor + unit)];
             const uint32_t s = it % S, ph = (it / S) & 1;
             ok = mbar_wait(empty0 + 8 * s, ph ^ 1, status, 1u);
             if (!ok) break;
@@ -293,14 +319,29 @@ eco_stream_kernel(const TensorDesc* __restrict__ descs, const uint32_t* __restri
                 reinterpret_cast<float*>(st + SL::kScales)[lane] = load_scale(T.scale, row0 + lane, bf16_scale);
             __syncwarp();
             if (lane == 0) mbar_arrive(full);
-            ++issued;
+            ++it;
+        }
+        if (lane == 0 && atomicAdd(tickets + 1, 1u) == gridDim.x - 1) {
+            tickets[0] = 0u;                               // every CTA has drawn its last ticket
+            tickets[1] = 0u;
+        }
+        if (ok) {
+            // end marker: a stage whose header says "no rows"
+            const uint32_t s = it % S, ph = (it / S) & 1;
+            ok = mbar_wait(empty0 + 8 * s, ph ^ 1, status, 1u);
+            if (ok && lane == 0) {
+                uint8_t* st = stage0 + static_cast<size_t>(s) * SL::kBytes;
+                reinterpret_cast<StageHeader*>(st + SL::kHeader)->nrows = 0u;
+                mbar_arrive_expect_tx(full0 + 8 * s, 0u);
+                mbar_arrive(full0 + 8 * s);
+            }
         }
         if (!ok) {
             // leave only after the copies already issued have landed (bounded)
-            const uint32_t pending = issued < static_cast<uint32_t>(S) ? issued : static_cast<uint32_t>(S);
+            const uint32_t pending = it < static_cast<uint32_t>(S) ? it : static_cast<uint32_t>(S);
             for (uint32_t k = 0; k < pending; ++k) {
-                const uint32_t it = issued - 1 - k;
-                mbar_wait(full0 + 8 * (it % S), (it / S) & 1, status, 2u);
+                const uint32_t j = it - 1 - k;
+                mbar_wait(full0 + 8 * (j % S), (j / S) & 1, status, 2u);
             }
         }
         return;
@@ -309,13 +350,15 @@ eco_stream_kernel(const TensorDesc* __restrict__ descs, const uint32_t* __restri
     // -------------------------------- consumers --------------------------------
     uint32_t cur_slot = 0xFFFFFFFFu;
     float run_max = 0.0f;                         // MODE_TENSOR_AMAX
-    for (uint32_t it = 0; it < n_my; ++it) {
+    for (uint32_t it = 0;; ++it) {
         const uint32_t s = it % S, ph = (it / S) & 1;
         if (!mbar_wait(full0 + 8 * s, ph, status, 3u)) return;
         const uint8_t* st = stage0 + static_cast<size_t>(s) * SL::kBytes;
         const StageHeader* h = reinterpret_cast<const StageHeader*>(st + SL::kHeader);
         const uint32_t empty = empty0 + 8 * s;
-        if (h->nrows == kUnitRows)
+        const uint32_t nrows = h->nrows;
+        if (nrows == 0u) break;                   // end marker
+        if (nrows == kUnitRows)
             consume_unit<FMT, OPT, RND, MODE, true>(P, bf16_scale, st, h, empty, warp, lane, scratch_amax, cur_slot, run_max);
         else
             consume_unit<FMT, OPT, RND, MODE, false>(P, bf16_scale, st, h, empty, warp, lane, scratch_amax, cur_slot, run_max);
@@ -330,7 +373,7 @@ eco_stream_kernel(const TensorDesc* __restrict__ descs, const uint32_t* __restri
 template <int FMT, int OPT, int RND, int MODE>
 static cudaError_t launch_one(const TensorDesc* descs, const uint32_t* unit_tensor, uint32_t n_units, const StepParams& P,
                               int bf16_scale, uint32_t* amax, uint32_t* amax_next, float* s_old, bool reverse,
-                              uint32_t* status, int grid_cap, cudaStream_t stream) {
+                              uint32_t* tickets, uint32_t* status, int grid_cap, cudaStream_t stream) {
     using SL = StageLayout<FMT, OPT>;
     static bool configured = false;
     auto kernel = eco_stream_kernel<FMT, OPT, RND, MODE>;
@@ -341,7 +384,7 @@ static cudaError_t launch_one(const TensorDesc* descs, const uint32_t* unit_tens
     }
     const uint32_t grid = n_units < static_cast<uint32_t>(grid_cap) ? n_units : static_cast<uint32_t>(grid_cap);
     kernel<<<grid, kStreamThreads, SL::kSmem, stream>>>(descs, unit_tensor, n_units, P, bf16_scale, amax, amax_next,
-                                                        s_old, reverse ? 1 : 0, status);
+                                                        s_old, reverse ? 1 : 0, MODE == MODE_BLOCK ? kInterleave : 1, tickets, status);
     return cudaGetLastError();
 }
 
@@ -357,20 +400,20 @@ static cudaError_t launch_one(const TensorDesc* descs, const uint32_t* unit_tens
 
 cudaError_t launch_stream(const LaunchConfig& c, int mode, const TensorDesc* descs, const uint32_t* unit_tensor,
                           uint32_t n_units, const StepParams& P, uint32_t* amax, uint32_t* amax_next, float* s_old,
-                          bool reverse, uint32_t* status, int grid_cap, cudaStream_t stream) {
+                          bool reverse, uint32_t* tickets, uint32_t* status, int grid_cap, cudaStream_t stream) {
     if (n_units == 0) return cudaSuccess;
     if (mode == STREAM_TENSOR_AMAX) {
         ECO_S_FMT(c.format, ECO_S_OPT(c.optimizer, {
             return launch_one<F, O, RND_RTN, MODE_TENSOR_AMAX>(descs, unit_tensor, n_units, P, c.bf16_scale, amax,
-                                                               amax_next, s_old, reverse, status, grid_cap, stream);
+                                                               amax_next, s_old, reverse, tickets, status, grid_cap, stream);
         }))
     }
     ECO_S_FMT(c.format, ECO_S_OPT(c.optimizer, ECO_S_RND(c.rounding, {
         if (mode == STREAM_BLOCK)
             return launch_one<F, O, R, MODE_BLOCK>(descs, unit_tensor, n_units, P, c.bf16_scale, amax, amax_next, s_old,
-                                                   reverse, status, grid_cap, stream);
+                                                   reverse, tickets, status, grid_cap, stream);
         return launch_one<F, O, R, MODE_TENSOR_APPLY>(descs, unit_tensor, n_units, P, c.bf16_scale, amax, amax_next,
-                                                      s_old, reverse, status, grid_cap, stream);
+                                                      s_old, reverse, tickets, status, grid_cap, stream);
     })))
     return cudaErrorInvalidValue;
 }
