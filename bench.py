@@ -6,7 +6,7 @@
 One "step" is one eco_step over every tensor of the workload's parameter set (the whole hot path:
 dequantize, optimizer update, amax/scale, requantize with stochastic rounding, error injection, stores).
 Prints ONE JSON line.  `value` = parameters updated per second with the state resident in HBM, timed
-with CUDA events on the launching stream; `e2e` = the same metric through eco_step_host with the state
+with CUDA events on the launching stream; `e2e` = the same metric through eco_host_step with the state
 in pinned HOST memory (copies inside the timed region).  With torchrun (N > 1) every rank steps its own
 replica of the parameter set (no data-path collective exists in this method) and the time is the max
 over ranks.  `--impl reference` times the CPU oracle instead (rank 0 only).
@@ -188,7 +188,8 @@ def run_reference(args):
 
 
 def run_e2e(w, device: int, steps: int, max_host_gb: float):
-    """eco_step_host on pinned host buffers: H2D of codes/scales/grads/moments, step, D2H of the results."""
+    """eco_host_step on pinned host buffers: every step copies codes/scales/grads/moments to the device, runs the
+    kernels and copies codes/scales/moments back (all inside the timed region)."""
     import torch
     from dataclasses import replace
     from paper_2601_22101_b200 import eco, workloads as wl
@@ -214,13 +215,15 @@ def run_e2e(w, device: int, steps: int, max_host_gb: float):
         tensors.append(eco.Tensor(cw, cs, cg, cm, cv, t.rows, t.cols, t.tensor_id))
     cfg = config_of(ws)
     up = down = 0
-    eco.eco_step_host(cfg, tensors, w.lr, w.beta1, w.beta2, w.eps, 1, w.step_seed, device)   # warm-up
+    handle = eco.eco_host_create(cfg, tensors, device)
+    eco.eco_host_step(handle, w.lr, w.beta1, w.beta2, w.eps, 1, w.step_seed)   # warm-up
     torch.cuda.synchronize(device)
     t0 = time.perf_counter()
     for s in range(steps):
-        up, down = eco.eco_step_host(cfg, tensors, w.lr, w.beta1, w.beta2, w.eps, 2 + s, w.step_seed, device)
+        up, down = eco.eco_host_step(handle, w.lr, w.beta1, w.beta2, w.eps, 2 + s, w.step_seed)
     torch.cuda.synchronize(device)
     el = time.perf_counter() - t0
+    eco.eco_host_destroy(handle)
     return {"value": ws.numel * steps / el, "unit": UNIT, "h2d_bytes_per_step": up, "d2h_bytes_per_step": down,
             "steps": steps, "params_per_step": ws.numel, "seconds": el,
             "sample": f"first {len(picked)} of {len(w.tensors)} tensors per GPU held in pinned host memory"}
@@ -231,13 +234,13 @@ def main():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=5)
-    ap.add_argument("--workload", default="c4", choices=["c1", "c2", "c3", "c4", "c5", "c3s", "c4s", "c5s"])
+    ap.add_argument("--workload", default="c4", choices=["c1", "c2", "c3", "c4", "c5", "c3r", "c3s", "c4s", "c5s"])
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--also", default="c3,c5", help="comma-separated workloads timed after the headline one and "
                     "reported under other_workloads (device-resident timing only)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--e2e-steps", type=int, default=2)
+    ap.add_argument("--e2e-steps", type=int, default=5)
     ap.add_argument("--e2e-host-gb", type=float, default=8.0)
     ap.add_argument("--option", action="append", default=[], help="name=value passed to eco_set_option")
     args = ap.parse_args()

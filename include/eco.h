@@ -25,6 +25,7 @@ extern "C" {
 #endif
 
 typedef struct eco_ctx eco_ctx;
+typedef struct eco_host_ctx eco_host_ctx;
 
 typedef enum eco_status {
     ECO_OK = 0,
@@ -127,16 +128,27 @@ eco_status eco_step(eco_ctx* ctx, float lr, float beta1, float beta2, float eps,
                     uint64_t step, uint64_t seed, void* cuda_stream);
 
 /*
- * eco_step_host -- the same step for callers that keep the state in HOST
- * memory (offloaded optimizer state).  `tensors` has the layout of eco_tensor
- * but every pointer is a host pointer (pinned memory makes the copies
- * asynchronous and faster).  Per tensor group the call copies codes, scales,
- * gradient and moments to device staging buffers it allocates, runs the
- * kernels of eco_step, copies codes, scales and moments back, and returns
- * after synchronizing its internal streams.  h2d_bytes / d2h_bytes (host,
- * optional) receive the bytes copied in each direction.
- * Errors: as eco_create and eco_step; ECO_ERR_NOMEM if staging cannot be allocated.
+ * eco_host_create / eco_host_step / eco_host_destroy -- the step of eco_step (Algorithm 1) for callers
+ * that keep the state in HOST memory (offloaded optimizer state).  `tensors` has the layout of
+ * eco_tensor but every pointer is a host pointer that must stay valid until eco_host_destroy (pinned
+ * memory makes the copies asynchronous and several times faster).
+ *   eco_host_create  cuts the list into chunks of whole tensors (about 256 MB of state), allocates three
+ *                    device staging slots of the largest chunk's size, three streams, and one eco_ctx per
+ *                    chunk.  Errors: as eco_create (the pointers are not required to be device memory).
+ *   eco_host_step    for every chunk: copies codes, scales, gradient and moments to its slot, runs the
+ *                    kernels of eco_step, copies codes, scales and moments back.  While one chunk is
+ *                    stepped the next is copied in and the previous one copied out, so both directions
+ *                    of the host link are busy at once.  Returns after everything has been copied back
+ *                    and the device-side status of every chunk has been checked.  h2d_bytes / d2h_bytes
+ *                    (host, optional) receive the bytes copied in each direction.  The gradient buffers
+ *                    are read at every call.  Errors: as eco_step, plus ECO_ERR_TIMEOUT.
+ *   eco_host_destroy frees all of it (synchronizes the device).  NULL is allowed.
+ * eco_step_host is the one-shot form: create, one step, destroy.
  */
+eco_status eco_host_create(eco_host_ctx** out, const eco_config* cfg, const eco_tensor* tensors, size_t n, int device);
+eco_status eco_host_step(eco_host_ctx* ctx, float lr, float beta1, float beta2, float eps, uint64_t step, uint64_t seed,
+                         uint64_t* h2d_bytes, uint64_t* d2h_bytes);
+eco_status eco_host_destroy(eco_host_ctx* ctx);
 eco_status eco_step_host(const eco_config* cfg, const eco_tensor* tensors, size_t n, int device,
                          float lr, float beta1, float beta2, float eps, uint64_t step, uint64_t seed,
                          uint64_t* h2d_bytes, uint64_t* d2h_bytes);
@@ -213,8 +225,8 @@ eco_status eco_quantize(const eco_config* cfg, const float* x, int64_t rows, int
 /*
  * eco_set_option -- process-wide tuning knobs read by the NEXT eco_create:
  *   "l2_group_bytes"  per-tensor scales only: bytes of inputs one pass-1/pass-2 launch pair
- *                     covers, so that pass 2 re-reads from L2 (-1 = half the L2 size, the
- *                     default; 0 = one pair for the whole context)
+ *                     covers (0, the default: one pair for the whole context, which measured
+ *                     fastest; -1 = half the L2 size, so that pass 2 re-reads from L2)
  *   "reverse_pass2"   per-tensor scales only: 1 (default) walks pass 2 in the opposite order
  *                     of pass 1 so that it starts with the most recently read data
  *   "use_stream"      1 (default) uses the persistent kernels fed by bulk asynchronous copies

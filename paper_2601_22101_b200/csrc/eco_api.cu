@@ -34,7 +34,7 @@ struct Launch {
 
 // Options settable through eco_set_option before eco_create.
 struct Options {
-    int64_t l2_group_bytes = -1;   // per-tensor scale: input bytes per launch pair; -1 = half of the L2 size, 0 = one group
+    int64_t l2_group_bytes = 0;    // per-tensor scale: input bytes per launch pair; -1 = half of the L2 size, 0 = one group
     int64_t reverse_pass2 = 1;     // per-tensor scale: walk pass 2 in the opposite order of pass 1
     int64_t use_stream = 1;        // 1: TMA-fed persistent kernels where the layout allows; 0: direct-load kernels only
     int64_t ctas_per_sm = 2;       // persistent grid = ctas_per_sm * SM count
@@ -506,12 +506,49 @@ eco_status eco_quantize(const eco_config* cfg, const float* x, int64_t rows, int
     return ECO_OK;
 }
 
-eco_status eco_step_host(const eco_config* cfg, const eco_tensor* tensors, size_t n, int device,
-                         float lr, float beta1, float beta2, float eps, uint64_t step, uint64_t seed,
-                         uint64_t* h2d_bytes, uint64_t* d2h_bytes) {
+}  // extern "C"
+
+// State held in HOST memory: the tensor list is cut into chunks of whole tensors (about 256 MB of state
+// each) that move through three device slots.  While chunk i is stepped, chunk i+1 is copied in and chunk
+// i-1 is copied out, so both directions of the host link stay busy.  Every buffer inside a slot is
+// 256-byte aligned.  Each chunk has its own eco_ctx bound to the slot it will occupy.
+struct eco_host_ctx {
+    struct Place { uint64_t w, scale, grad, m, v, wb, sb, gb, mb; };
+    struct Chunk { size_t first, count; uint64_t bytes; };
+    eco_config cfg;
+    int device = 0;
+    bool adam = false;
+    std::vector<eco_tensor> host, dev;
+    std::vector<Place> place;
+    std::vector<Chunk> chunks;
+    std::vector<eco_ctx*> ctxs;
+    std::vector<cudaEvent_t> ev_in, ev_run, ev_out;
+    cudaStream_t s_in = nullptr, s_run = nullptr, s_out = nullptr;
+    uint8_t* arena = nullptr;
+    uint64_t slot_bytes = 0, up = 0, down = 0;
+    int n_slots = 0;
+};
+
+extern "C" {
+
+eco_status eco_host_destroy(eco_host_ctx* h) {
+    if (!h) return ECO_OK;
+    cudaSetDevice(h->device);
+    for (eco_ctx* c : h->ctxs) if (c) eco_destroy(c);
+    for (auto* v : {&h->ev_in, &h->ev_run, &h->ev_out}) for (cudaEvent_t e : *v) if (e) cudaEventDestroy(e);
+    if (h->s_in) cudaStreamDestroy(h->s_in);
+    if (h->s_run) cudaStreamDestroy(h->s_run);
+    if (h->s_out) cudaStreamDestroy(h->s_out);
+    cudaFree(h->arena);
+    delete h;
+    return ECO_OK;
+}
+
+eco_status eco_host_create(eco_host_ctx** out, const eco_config* cfg, const eco_tensor* tensors, size_t n, int device) {
+    if (!out) return fail(nullptr, ECO_ERR_INVALID_ARG, "out is NULL");
+    *out = nullptr;
     if (eco_status st = check_config(cfg, true)) return st;
     if (!tensors || n == 0) return fail(nullptr, ECO_ERR_INVALID_ARG, "empty tensor list");
-    if (eco_status st = check_hyper(nullptr, *cfg, lr, beta1, beta2, eps, step)) return st;
     const bool adam = cfg->optimizer == ECO_OPT_ADAM;
     for (size_t i = 0; i < n; ++i) {
         const eco_tensor& t = tensors[i];
@@ -520,74 +557,139 @@ eco_status eco_step_host(const eco_config* cfg, const eco_tensor* tensors, size_
             return fail(nullptr, ECO_ERR_INVALID_ARG, "tensor %zu: NULL buffer (or v given for SGDM)", i);
     }
     ECO_CUDA(nullptr, cudaSetDevice(device));
-
-    // Device staging: one arena, every buffer 256-byte aligned.
+    eco_host_ctx* h = new (std::nothrow) eco_host_ctx;
+    if (!h) return fail(nullptr, ECO_ERR_NOMEM, "out of host memory");
+    h->cfg = *cfg;
+    h->device = device;
+    h->adam = adam;
+    h->host.assign(tensors, tensors + n);
+    h->dev.assign(tensors, tensors + n);
+    h->place.resize(n);
     auto align = [](uint64_t x) { return (x + 255) & ~uint64_t(255); };
-    struct Stage { uint64_t w, scale, grad, m, v, wb, sb, gb, mb; };
-    std::vector<Stage> st(n);
-    uint64_t total = 0;
-    for (size_t i = 0; i < n; ++i) {
-        const uint64_t numel = static_cast<uint64_t>(tensors[i].rows) * static_cast<uint64_t>(tensors[i].cols);
-        Stage& s = st[i];
-        s.wb = code_bytes(*cfg, numel); s.sb = scale_bytes(*cfg, tensors[i].rows, tensors[i].cols);
-        s.gb = numel * 2; s.mb = numel * 4;
-        s.w = total; total += align(s.wb);
-        s.scale = total; total += align(s.sb);
-        s.grad = total; total += align(s.gb);
-        s.m = total; total += align(s.mb);
-        s.v = total; if (adam) total += align(s.mb);
+    constexpr uint64_t kChunkTarget = 256ull << 20;
+    constexpr int kSlots = 3;
+    {
+        eco_host_ctx::Chunk c{0, 0, 0};
+        for (size_t i = 0; i < n; ++i) {
+            const uint64_t numel = static_cast<uint64_t>(tensors[i].rows) * static_cast<uint64_t>(tensors[i].cols);
+            eco_host_ctx::Place& p = h->place[i];
+            p.wb = code_bytes(*cfg, numel); p.sb = scale_bytes(*cfg, tensors[i].rows, tensors[i].cols);
+            p.gb = numel * 2; p.mb = numel * 4;
+            const uint64_t need = align(p.wb) + align(p.sb) + align(p.gb) + align(p.mb) * (adam ? 2 : 1);
+            if (c.count > 0 && c.bytes + need > kChunkTarget) {
+                h->chunks.push_back(c);
+                c = eco_host_ctx::Chunk{i, 0, 0};
+            }
+            uint64_t off = c.bytes;
+            p.w = off; off += align(p.wb);
+            p.scale = off; off += align(p.sb);
+            p.grad = off; off += align(p.gb);
+            p.m = off; off += align(p.mb);
+            p.v = off; if (adam) off += align(p.mb);
+            c.bytes = off;
+            c.count++;
+            h->slot_bytes = std::max(h->slot_bytes, c.bytes);
+        }
+        h->chunks.push_back(c);
     }
-    uint8_t* arena = nullptr;
-    ECO_CUDA(nullptr, cudaMalloc(&arena, total));
-    cudaStream_t stream = nullptr;
-    eco_ctx* ctx = nullptr;
-    eco_status rc = ECO_OK;
-    uint64_t up = 0, down = 0;
-    std::vector<eco_tensor> dev(n);
-    auto bail = [&](eco_status s) {
-        if (ctx) eco_destroy(ctx);
-        if (stream) cudaStreamDestroy(stream);
-        cudaFree(arena);
-        return s;
-    };
+    h->n_slots = static_cast<int>(std::min<size_t>(kSlots, h->chunks.size()));
+    const size_t nc = h->chunks.size();
+    h->ctxs.assign(nc, nullptr);
+    h->ev_in.assign(nc, nullptr); h->ev_run.assign(nc, nullptr); h->ev_out.assign(nc, nullptr);
 #define ECO_CUDA_H(call)                                                                             \
     do {                                                                                             \
         cudaError_t e_ = (call);                                                                     \
-        if (e_ != cudaSuccess) return bail(fail(nullptr, ECO_ERR_CUDA, "%s failed: %s", #call, cudaGetErrorString(e_))); \
+        if (e_ != cudaSuccess) {                                                                     \
+            eco_status st_ = fail(nullptr, e_ == cudaErrorMemoryAllocation ? ECO_ERR_NOMEM : ECO_ERR_CUDA, \
+                                  "%s failed: %s", #call, cudaGetErrorString(e_));                   \
+            eco_host_destroy(h);                                                                     \
+            return st_;                                                                              \
+        }                                                                                            \
     } while (0)
-    ECO_CUDA_H(cudaStreamCreateWithFlags(&stream, cudaStreamNonBlocking));
-    for (size_t i = 0; i < n; ++i) {
-        const Stage& s = st[i];
-        dev[i] = tensors[i];
-        dev[i].w = arena + s.w;
-        dev[i].scale = arena + s.scale;
-        dev[i].grad = arena + s.grad;
-        dev[i].m = reinterpret_cast<float*>(arena + s.m);
-        dev[i].v = adam ? reinterpret_cast<float*>(arena + s.v) : nullptr;
-        ECO_CUDA_H(cudaMemcpyAsync(dev[i].w, tensors[i].w, s.wb, cudaMemcpyHostToDevice, stream));
-        ECO_CUDA_H(cudaMemcpyAsync(dev[i].scale, tensors[i].scale, s.sb, cudaMemcpyHostToDevice, stream));
-        ECO_CUDA_H(cudaMemcpyAsync(const_cast<void*>(dev[i].grad), tensors[i].grad, s.gb, cudaMemcpyHostToDevice, stream));
-        ECO_CUDA_H(cudaMemcpyAsync(dev[i].m, tensors[i].m, s.mb, cudaMemcpyHostToDevice, stream));
-        up += s.wb + s.sb + s.gb + s.mb;
-        if (adam) { ECO_CUDA_H(cudaMemcpyAsync(dev[i].v, tensors[i].v, s.mb, cudaMemcpyHostToDevice, stream)); up += s.mb; }
+    ECO_CUDA_H(cudaMalloc(&h->arena, h->slot_bytes * h->n_slots));
+    ECO_CUDA_H(cudaStreamCreateWithFlags(&h->s_in, cudaStreamNonBlocking));
+    ECO_CUDA_H(cudaStreamCreateWithFlags(&h->s_run, cudaStreamNonBlocking));
+    ECO_CUDA_H(cudaStreamCreateWithFlags(&h->s_out, cudaStreamNonBlocking));
+    for (size_t c = 0; c < nc; ++c) {
+        uint8_t* base = h->arena + h->slot_bytes * (c % h->n_slots);
+        for (size_t i = h->chunks[c].first; i < h->chunks[c].first + h->chunks[c].count; ++i) {
+            const eco_host_ctx::Place& p = h->place[i];
+            h->dev[i].w = base + p.w;
+            h->dev[i].scale = base + p.scale;
+            h->dev[i].grad = base + p.grad;
+            h->dev[i].m = reinterpret_cast<float*>(base + p.m);
+            h->dev[i].v = adam ? reinterpret_cast<float*>(base + p.v) : nullptr;
+        }
+        eco_status rc = eco_create(&h->ctxs[c], cfg, h->dev.data() + h->chunks[c].first, h->chunks[c].count, device);
+        if (rc != ECO_OK) { eco_host_destroy(h); return rc; }
+        ECO_CUDA_H(cudaEventCreateWithFlags(&h->ev_in[c], cudaEventDisableTiming));
+        ECO_CUDA_H(cudaEventCreateWithFlags(&h->ev_run[c], cudaEventDisableTiming));
+        ECO_CUDA_H(cudaEventCreateWithFlags(&h->ev_out[c], cudaEventDisableTiming));
     }
-    rc = eco_create(&ctx, cfg, dev.data(), n, device);
-    if (rc != ECO_OK) return bail(rc);
-    rc = eco_step(ctx, lr, beta1, beta2, eps, step, seed, stream);
-    if (rc != ECO_OK) { g_thread_error = ctx->err; return bail(rc); }
-    for (size_t i = 0; i < n; ++i) {
-        const Stage& s = st[i];
-        ECO_CUDA_H(cudaMemcpyAsync(tensors[i].w, dev[i].w, s.wb, cudaMemcpyDeviceToHost, stream));
-        ECO_CUDA_H(cudaMemcpyAsync(tensors[i].scale, dev[i].scale, s.sb, cudaMemcpyDeviceToHost, stream));
-        ECO_CUDA_H(cudaMemcpyAsync(tensors[i].m, dev[i].m, s.mb, cudaMemcpyDeviceToHost, stream));
-        down += s.wb + s.sb + s.mb;
-        if (adam) { ECO_CUDA_H(cudaMemcpyAsync(tensors[i].v, dev[i].v, s.mb, cudaMemcpyDeviceToHost, stream)); down += s.mb; }
-    }
-    ECO_CUDA_H(cudaStreamSynchronize(stream));
 #undef ECO_CUDA_H
+    *out = h;
+    return ECO_OK;
+}
+
+eco_status eco_host_step(eco_host_ctx* h, float lr, float beta1, float beta2, float eps, uint64_t step, uint64_t seed,
+                         uint64_t* h2d_bytes, uint64_t* d2h_bytes) {
+    if (!h) return fail(nullptr, ECO_ERR_INVALID_ARG, "ctx is NULL");
+    if (eco_status st = check_hyper(nullptr, h->cfg, lr, beta1, beta2, eps, step)) return st;
+    ECO_CUDA(nullptr, cudaSetDevice(h->device));
+    const bool adam = h->adam;
+    uint64_t up = 0, down = 0;
+    for (size_t c = 0; c < h->chunks.size(); ++c) {
+        const size_t first = h->chunks[c].first, last = first + h->chunks[c].count;
+        // the slot is free once the chunk that used it before has been copied out
+        if (c >= static_cast<size_t>(h->n_slots)) ECO_CUDA(nullptr, cudaStreamWaitEvent(h->s_in, h->ev_out[c - h->n_slots], 0));
+        for (size_t i = first; i < last; ++i) {
+            const eco_host_ctx::Place& p = h->place[i];
+            const eco_tensor &src = h->host[i], &dst = h->dev[i];
+            ECO_CUDA(nullptr, cudaMemcpyAsync(dst.w, src.w, p.wb, cudaMemcpyHostToDevice, h->s_in));
+            ECO_CUDA(nullptr, cudaMemcpyAsync(dst.scale, src.scale, p.sb, cudaMemcpyHostToDevice, h->s_in));
+            ECO_CUDA(nullptr, cudaMemcpyAsync(const_cast<void*>(dst.grad), src.grad, p.gb, cudaMemcpyHostToDevice, h->s_in));
+            ECO_CUDA(nullptr, cudaMemcpyAsync(dst.m, src.m, p.mb, cudaMemcpyHostToDevice, h->s_in));
+            up += p.wb + p.sb + p.gb + p.mb;
+            if (adam) { ECO_CUDA(nullptr, cudaMemcpyAsync(dst.v, src.v, p.mb, cudaMemcpyHostToDevice, h->s_in)); up += p.mb; }
+        }
+        ECO_CUDA(nullptr, cudaEventRecord(h->ev_in[c], h->s_in));
+        ECO_CUDA(nullptr, cudaStreamWaitEvent(h->s_run, h->ev_in[c], 0));
+        eco_status rc = eco_step(h->ctxs[c], lr, beta1, beta2, eps, step, seed, h->s_run);
+        if (rc != ECO_OK) { g_thread_error = h->ctxs[c]->err; cudaDeviceSynchronize(); return rc; }
+        ECO_CUDA(nullptr, cudaEventRecord(h->ev_run[c], h->s_run));
+        ECO_CUDA(nullptr, cudaStreamWaitEvent(h->s_out, h->ev_run[c], 0));
+        for (size_t i = first; i < last; ++i) {
+            const eco_host_ctx::Place& p = h->place[i];
+            const eco_tensor &dst = h->host[i], &src = h->dev[i];
+            ECO_CUDA(nullptr, cudaMemcpyAsync(dst.w, src.w, p.wb, cudaMemcpyDeviceToHost, h->s_out));
+            ECO_CUDA(nullptr, cudaMemcpyAsync(dst.scale, src.scale, p.sb, cudaMemcpyDeviceToHost, h->s_out));
+            ECO_CUDA(nullptr, cudaMemcpyAsync(dst.m, src.m, p.mb, cudaMemcpyDeviceToHost, h->s_out));
+            down += p.wb + p.sb + p.mb;
+            if (adam) { ECO_CUDA(nullptr, cudaMemcpyAsync(dst.v, src.v, p.mb, cudaMemcpyDeviceToHost, h->s_out)); down += p.mb; }
+        }
+        ECO_CUDA(nullptr, cudaEventRecord(h->ev_out[c], h->s_out));
+    }
+    ECO_CUDA(nullptr, cudaStreamSynchronize(h->s_out));
+    ECO_CUDA(nullptr, cudaStreamSynchronize(h->s_in));
+    for (eco_ctx* c : h->ctxs) {
+        eco_status rc = eco_check(c, h->s_run);
+        if (rc != ECO_OK) { g_thread_error = c->err; return rc; }
+    }
     if (h2d_bytes) *h2d_bytes = up;
     if (d2h_bytes) *d2h_bytes = down;
-    return bail(ECO_OK);
+    return ECO_OK;
+}
+
+eco_status eco_step_host(const eco_config* cfg, const eco_tensor* tensors, size_t n, int device,
+                         float lr, float beta1, float beta2, float eps, uint64_t step, uint64_t seed,
+                         uint64_t* h2d_bytes, uint64_t* d2h_bytes) {
+    if (eco_status st = check_config(cfg, true)) return st;
+    if (eco_status st = check_hyper(nullptr, *cfg, lr, beta1, beta2, eps, step)) return st;
+    eco_host_ctx* h = nullptr;
+    if (eco_status st = eco_host_create(&h, cfg, tensors, n, device)) return st;
+    const eco_status st = eco_host_step(h, lr, beta1, beta2, eps, step, seed, h2d_bytes, d2h_bytes);
+    eco_host_destroy(h);
+    return st;
 }
 
 // ---------------------------------------------------------------------------

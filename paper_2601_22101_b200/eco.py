@@ -24,7 +24,8 @@ ECO_OPT_SGDM, ECO_OPT_ADAM = 0, 1
 ECO_ROUND_NEAREST, ECO_ROUND_STOCHASTIC = 0, 1
 ECO_INJECT_NONE, ECO_INJECT_ECO = 0, 1
 
-EXPORTED = ("eco_create", "eco_step", "eco_step_host", "eco_step_static", "eco_check", "eco_destroy", "eco_last_error", "eco_quantize",
+EXPORTED = ("eco_create", "eco_step", "eco_step_host", "eco_host_create", "eco_host_step", "eco_host_destroy",
+            "eco_step_static", "eco_check", "eco_destroy", "eco_last_error", "eco_quantize",
             "eco_set_option", "eco_num_launches", "eco_version")
 
 
@@ -67,6 +68,13 @@ def load_library() -> ctypes.CDLL:
         L.eco_step_host.argtypes = [ctypes.POINTER(eco_config), ctypes.POINTER(eco_tensor), ctypes.c_size_t,
                                     ctypes.c_int, f32, f32, f32, f32, u64, u64,
                                     ctypes.POINTER(u64), ctypes.POINTER(u64)]
+        L.eco_host_create.restype = ctypes.c_int
+        L.eco_host_create.argtypes = [ctypes.POINTER(vp), ctypes.POINTER(eco_config), ctypes.POINTER(eco_tensor),
+                                      ctypes.c_size_t, ctypes.c_int]
+        L.eco_host_step.restype = ctypes.c_int
+        L.eco_host_step.argtypes = [vp, f32, f32, f32, f32, u64, u64, ctypes.POINTER(u64), ctypes.POINTER(u64)]
+        L.eco_host_destroy.restype = ctypes.c_int
+        L.eco_host_destroy.argtypes = [vp]
         L.eco_step_static.restype = ctypes.c_int
         L.eco_step_static.argtypes = [ctypes.POINTER(eco_config), ctypes.POINTER(eco_tensor), ctypes.c_size_t,
                                       ctypes.c_int, f32, f32, f32, f32, u64, u64, vp]
@@ -170,6 +178,32 @@ def eco_step_host(cfg: Config, tensors: Sequence[Tensor], lr: float, beta1: floa
     if st != ECO_OK:
         _raise(st)
     return up.value, down.value
+
+
+def eco_host_create(cfg: Config, tensors: Sequence[Tensor], device: int = 0) -> int:
+    """Bind a list of HOST buffers for repeated host-resident steps; returns the handle.  The buffers must
+    stay alive until ``eco_host_destroy``.  See include/eco.h."""
+    L = load_library()
+    handle = ctypes.c_void_p()
+    c = cfg.c()
+    arr = _tensor_array(tensors)
+    st = L.eco_host_create(ctypes.byref(handle), ctypes.byref(c), arr, len(tensors), device)
+    if st != ECO_OK:
+        _raise(st)
+    return handle.value
+
+
+def eco_host_step(handle: int, lr: float, beta1: float, beta2: float, eps: float, step: int, seed: int):
+    """One step on the host-resident state bound by ``eco_host_create``; returns (h2d_bytes, d2h_bytes)."""
+    up, down = ctypes.c_uint64(), ctypes.c_uint64()
+    st = load_library().eco_host_step(handle, lr, beta1, beta2, eps, step, seed, ctypes.byref(up), ctypes.byref(down))
+    if st != ECO_OK:
+        _raise(st)
+    return up.value, down.value
+
+
+def eco_host_destroy(handle: int) -> None:
+    load_library().eco_host_destroy(handle)
 
 
 def eco_step_static(cfg: Config, tensors: Sequence[Tensor], lr: float, beta1: float, beta2: float, eps: float,

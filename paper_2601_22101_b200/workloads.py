@@ -199,6 +199,12 @@ def c3_small() -> Workload:
     return replace(w, name=w.name + "_small")
 
 
+def c3_rowwise() -> Workload:
+    """The Gemma-3-1B-shaped set with one FP8 scale per row: the granularity of the paper's own FP8 runs (Sec. 4.1)."""
+    w = c3()
+    return replace(w, name="c3_gemma3_1b_fp8_row_adam_sr", granularity=PER_ROW)
+
+
 def c4_small() -> Workload:
     """One layer (64 experts) of the sparse-MoE set (profiling-sized: ~1.5 GB of state)."""
     w = c4(layers=1)
@@ -241,7 +247,7 @@ def replicate(w: Workload, copies: int) -> Workload:
     return replace(w, name=f"{w.name}_x{copies}", tensors=ts)
 
 
-BY_NAME = {"c1": c1, "c2": c2, "c3": c3, "c4": c4, "c5": c5,
+BY_NAME = {"c1": c1, "c2": c2, "c3": c3, "c4": c4, "c5": c5, "c3r": c3_rowwise,
            "c3s": c3_small, "c4s": c4_small, "c5s": c5_small}
 
 

@@ -177,3 +177,60 @@ def test_checkpoint_resume_is_bit_exact():
         assert torch.equal(ta.w, tb.w) and torch.equal(ta.scale, tb.scale)
         assert torch.equal(ta.m, tb.m) and torch.equal(ta.v, tb.v)
     a.destroy(); b.destroy()
+
+
+def _host_tensors(w, dev):
+    """Host copies (torch CPU tensors) of a DeviceState's buffers, as eco.Tensor list."""
+    out = []
+    for t, d in zip(w.tensors, dev.tensors):
+        out.append(eco.Tensor(d.w.cpu(), d.scale.cpu(), d.grad.cpu(), d.m.cpu(), None if d.v is None else d.v.cpu(),
+                              t.rows, t.cols, t.tensor_id))
+    return out
+
+
+def test_step_host_small_ragged_against_oracle():
+    """eco_step_host (state in host memory) on ragged shapes, two chained steps, against the oracle."""
+    w = _mini(wl.FP8_E4M3, wl.PER_TENSOR, wl.SCALE_F32, wl.ADAM, wl.SR, RAGGED)
+    dev = DeviceState(w)
+    dev.init_from_host()
+    ora = OracleState(w)
+    host = _host_tensors(w, dev)
+    for step in (1, 2):
+        grads = [wl.gradient_bf16(w, t, step) for t in w.tensors]
+        for h, g in zip(host, grads):
+            h.grad.view(torch.int16).copy_(torch.from_numpy(g.view(np.int16)))
+        up, down = eco.eco_step_host(config_of(w), host, w.lr, w.beta1, w.beta2, w.eps, step, w.step_seed)
+        assert up > 0 and down > 0
+        ora.step(step, grads)
+        for i, h in enumerate(host):
+            assert (h.w.numpy() == ora.w[i]).all()
+            assert (h.scale.view(torch.int32).numpy() == ora.scale[i].view(np.int32)).all()
+            np.testing.assert_allclose(h.m.numpy(), ora.m[i], rtol=RTOL, atol=ATOL)
+            np.testing.assert_allclose(h.v.numpy(), ora.v[i], rtol=RTOL, atol=ATOL)
+
+
+def test_step_host_pipelined_chunks_match_device_resident_step():
+    """Several staging chunks in flight (each tensor is ~180 MB of state): same bits as the device-resident step."""
+    ts = [wl.TensorSpec(f"big{i}", 4096, 4096, 50 + i, zero_grad=(i == 1)) for i in range(4)]
+    w = wl.Workload("host_chunks", wl.FP8_E4M3, wl.PER_BLOCK, 128, wl.SCALE_F32, wl.ADAM, wl.SR, lr=1e-3, beta1=0.9,
+                    beta2=0.95, eps=1e-8, weight_std=0.02, grad_std=1e-3, steps=2, step_seed=99, tensors=ts)
+    dev = DeviceState(w)
+    dev.init_on_device(seed=5)
+    dev.set_grads_on_device(seed=6)
+    host = [eco.Tensor(h.w.pin_memory(), h.scale.pin_memory(), h.grad.pin_memory(), h.m.pin_memory(), h.v.pin_memory(),
+                       h.rows, h.cols, h.tensor_id) for h in _host_tensors(w, dev)]
+    dev.create()
+    handle = eco.eco_host_create(config_of(w), host)
+    try:
+        for step in (1, 2):
+            dev.step(step)
+            up, down = eco.eco_host_step(handle, w.lr, w.beta1, w.beta2, w.eps, step, w.step_seed)
+            assert up == sum(t.numel for t in ts) * 11 + sum(w.n_scales(t) for t in ts) * 4
+            assert down == sum(t.numel for t in ts) * 9 + sum(w.n_scales(t) for t in ts) * 4
+        torch.cuda.synchronize()
+        for d, h in zip(dev.tensors, host):
+            assert torch.equal(d.w.cpu(), h.w) and torch.equal(d.scale.cpu(), h.scale)
+            assert torch.equal(d.m.cpu(), h.m) and torch.equal(d.v.cpu(), h.v)
+    finally:
+        eco.eco_host_destroy(handle)
+        dev.destroy()
