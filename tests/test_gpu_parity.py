@@ -234,3 +234,69 @@ def test_step_host_pipelined_chunks_match_device_resident_step():
     finally:
         eco.eco_host_destroy(handle)
         dev.destroy()
+
+
+# ---------------------------------------------------------------------------------------------------
+# Full-size parameter sets in the launch configuration the benchmark times (one context over the whole
+# set, state drawn on the device), checked on SAMPLED WHOLE TENSORS: tensors never interact, so the
+# oracle can step any one of them alone from a copy of its inputs taken before the step.
+# ---------------------------------------------------------------------------------------------------
+def _sampled_full_size(w: wl.Workload, sample_ids, steps=2):
+    dev = DeviceState(w)
+    dev.init_on_device(seed=77)
+    dev.set_grads_on_device(seed=78)
+    cfg_o = oracle_config(w)
+    before = {}
+    for i in sample_ids:
+        d = dev.tensors[i]
+        before[i] = [d.w.cpu().numpy().copy(), _np(d.scale.view(torch.int16 if d.scale.dtype == torch.bfloat16 else torch.float32)).copy(),
+                     d.grad.view(torch.int16).cpu().numpy().view(np.uint16).copy(), d.m.cpu().numpy().copy(),
+                     None if d.v is None else d.v.cpu().numpy().copy()]
+        if w.scale_dtype == wl.SCALE_BF16:
+            before[i][1] = before[i][1].view(np.uint16)
+    dev.create()
+    try:
+        for step in range(1, steps + 1):
+            dev.step(step)
+        torch.cuda.synchronize()
+        eco.eco_check(dev.handle, torch.cuda.current_stream().cuda_stream)
+        for i in sample_ids:
+            t = w.tensors[i]
+            cw, cs, cg, cm, cv = before[i]
+            for step in range(1, steps + 1):
+                oracle.step(cfg_o, lr=float(np.float32(w.lr)), beta1=float(np.float32(w.beta1)), beta2=float(np.float32(w.beta2)),
+                            eps=float(np.float32(w.eps)), step=step, seed=w.step_seed, w=cw, scale=cs, grad=cg, m=cm, v=cv,
+                            rows=t.rows, cols=t.cols, tensor_id=t.tensor_id)
+            d = dev.tensors[i]
+            tag = f"{w.name} tensor {i} {t.name} [{t.rows}x{t.cols}]"
+            assert (_np(d.w) == cw).all(), tag + ": codes differ"
+            assert (_scale_bits(d.scale) == _oracle_scale_bits(cs)).all(), tag + ": scales differ"
+            np.testing.assert_allclose(_np(d.m), cm, rtol=RTOL, atol=ATOL, err_msg=tag + " m")
+            if cv is not None:
+                np.testing.assert_allclose(_np(d.v), cv, rtol=RTOL, atol=ATOL, err_msg=tag + " v")
+    finally:
+        dev.destroy()
+
+
+def _spread(n, k):
+    return sorted({int(round(j * (n - 1) / (k - 1))) for j in range(k)})
+
+
+def test_c4_full_size_sampled_tensors():
+    w = wl.c4()
+    ids = set(_spread(len(w.tensors), 24))
+    ids |= set([i for i, t in enumerate(w.tensors) if t.zero_grad][:: 200])      # make sure zero-gradient experts are in
+    _sampled_full_size(w, sorted(ids))
+
+
+def test_c3_full_size_sampled_tensors():
+    w = wl.c3()
+    n = len(w.tensors)
+    ids = list(range(7)) + list(range(n - 8, n - 1)) + [n - 1]        # first and last layer, and the 302M-parameter embedding
+    _sampled_full_size(w, ids, steps=1)
+
+
+def test_c5_full_size_sampled_tensors():
+    w = wl.c5()
+    ids = {0, 1, 2} | {3 + i for i in _spread(len(w.tensors) - 3, 18)}   # the dense layer (rows of 10944 = 85*128 + 64) + experts
+    _sampled_full_size(w, sorted(ids))
