@@ -31,7 +31,14 @@ FALLBACK_HBM_GBS = 6650.0
 # DRAM traffic per parameter of the dominant kernel from an ncu capture
 # (dram__bytes_read.sum + dram__bytes_write.sum over the launch, divided by its parameters);
 # sources are the summaries under profiles/.  None = not captured.
-NCU_DRAM_BYTES_PER_PARAM = {}
+NCU_DRAM_BYTES_PER_PARAM = {
+    # profiles/eco_stream_kernel_c4s.md: 1.4808 GB read + 1.1638 GB written over 134,217,728 parameters
+    "eco_stream_kernel<fp8,adam,sr,block>": 19.70,
+    # profiles/eco_stream_kernel_c5s.md: 1.1941 GB + 0.7723 GB over 183,304,192 parameters
+    "eco_stream_kernel<int4,sgdm,sr,block>": 10.73,
+    # profiles/eco_stream_kernel_c3s.md (apply pass): 1.0058 GB + 0.7672 GB over 91,422,720 parameters
+    "eco_stream_kernel<fp8,adam,sr,tensor_apply>": 19.39,
+}
 
 
 def _workload(name: str):
@@ -50,6 +57,20 @@ def _dominant_kernel(w) -> str:
         return f"eco_row_kernel<{fmt},{opt},{rnd}>"
     mode = "block" if w.granularity == wl.PER_BLOCK else "tensor_apply"
     return f"eco_stream_kernel<{fmt},{opt},{rnd},{mode}>"
+
+
+def _two_pass_note(w, params, ms_per_step, peak):
+    """Per-tensor scales need max|theta~| over a whole tensor before any element can be rounded, so a tensor
+    larger than the on-chip memories is read twice: the kernels move 11 + 11 + 9 = 31 B/param (FP8 + Adam)
+    where the method needs 20.  Reported beside the algorithmic figure so that both are visible."""
+    from paper_2601_22101_b200 import workloads as wl
+    if w.granularity != wl.PER_TENSOR:
+        return {}
+    code = 1.0 if w.format == wl.FP8_E4M3 else 0.5
+    moments = 4.0 * (2 if w.optimizer == wl.ADAM else 1)
+    moved = 2 * (code + 2.0 + moments) + (code + moments)
+    gbs = params * moved / (ms_per_step * 1e-3) / 1e9
+    return {"two_pass_bytes_per_param": moved, "two_pass_achieved": gbs, "two_pass_frac": gbs / peak}
 
 
 def _measured_peak():
@@ -320,7 +341,8 @@ def main():
                          "frac": achieved / peak, "peak_source": peak_src,
                          "frac_of_nominal_8000": achieved / 8000.0,
                          "algorithmic_bytes_per_param": bpp,
-                         "traffic": (tr * params_per_rank if tr else None)},
+                         "traffic": (tr * params_per_rank if tr else None),
+                         **_two_pass_note(w_global, params_per_rank, ms_per_step, peak)},
         }
 
     stream = torch.cuda.current_stream()
