@@ -53,9 +53,7 @@ def _dominant_kernel(w) -> str:
     fmt = "fp8" if w.format == wl.FP8_E4M3 else "int4"
     opt = "adam" if w.optimizer == wl.ADAM else "sgdm"
     rnd = "sr" if w.rounding == wl.SR else "rtn"
-    if w.granularity == wl.PER_ROW:
-        return f"eco_row_kernel<{fmt},{opt},{rnd}>"
-    mode = "block" if w.granularity == wl.PER_BLOCK else "tensor_apply"
+    mode = {wl.PER_BLOCK: "block", wl.PER_TENSOR: "tensor_apply", wl.PER_ROW: "row"}[w.granularity]
     return f"eco_stream_kernel<{fmt},{opt},{rnd},{mode}>"
 
 

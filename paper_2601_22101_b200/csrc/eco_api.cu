@@ -23,7 +23,8 @@ namespace {
 
 thread_local std::string g_thread_error;
 
-enum LaunchKind { KIND_BLOCK_FAST = 0, KIND_BLOCK_GENERIC = 1, KIND_TENSOR = 2, KIND_ROW = 3, KIND_TENSOR_STREAM = 4 };
+enum LaunchKind { KIND_BLOCK_FAST = 0, KIND_BLOCK_GENERIC = 1, KIND_TENSOR = 2, KIND_ROW = 3, KIND_TENSOR_STREAM = 4,
+                  KIND_ROW_STREAM = 5 };
 
 struct Launch {
     int kind;
@@ -309,6 +310,11 @@ eco_status eco_create(eco_ctx** out, const eco_config* cfg, const eco_tensor* te
             if (kind == KIND_ROW) {
                 d.n_blocks = static_cast<uint64_t>(tensors[members[k]].rows);
                 nu = d.n_blocks;
+            } else if (kind == KIND_ROW_STREAM) {
+                // a unit is as many whole matrix rows as fit 32 rows of 128 elements
+                d.n_blocks = static_cast<uint64_t>(tensors[members[k]].rows) * d.blocks_per_row;
+                d.unit_rows = (static_cast<uint32_t>(eco::stream_unit_rows()) / d.blocks_per_row) * d.blocks_per_row;
+                nu = (d.n_blocks + d.unit_rows - 1) / d.unit_rows;
             } else {
                 d.n_blocks = (kind == KIND_TENSOR || kind == KIND_TENSOR_STREAM) ? (d.numel + 127) / 128
                                                    : static_cast<uint64_t>(tensors[members[k]].rows) * d.blocks_per_row;
@@ -332,10 +338,14 @@ eco_status eco_create(eco_ctx** out, const eco_config* cfg, const eco_tensor* te
         ok = add_launch(KIND_BLOCK_FAST, fast) && add_launch(KIND_BLOCK_GENERIC, generic);
         ctx->num_launches = static_cast<int>(ctx->launches.size());
     } else if (cfg->granularity == ECO_SCALE_PER_ROW) {
-        std::vector<size_t> all(n);
-        for (size_t i = 0; i < n; ++i) all[i] = i;
-        ok = add_launch(KIND_ROW, all);
-        ctx->num_launches = 1;
+        // matrix rows of whole 128-element rows, at most 32 of them, go to the streaming kernel
+        std::vector<size_t> fast, generic;
+        for (size_t i = 0; i < n; ++i) {
+            const bool streams = use_stream && tensors[i].cols % 128 == 0 && tensors[i].cols / 128 <= eco::stream_unit_rows();
+            (streams ? fast : generic).push_back(i);
+        }
+        ok = add_launch(KIND_ROW_STREAM, fast) && add_launch(KIND_ROW, generic);
+        ctx->num_launches = static_cast<int>(ctx->launches.size());
     } else {
         // Per-tensor scale: pass 1 + pass 2 per group of tensors whose inputs fit the L2 budget, so
         // that pass 2 finds what pass 1 read still cached.
@@ -431,6 +441,10 @@ eco_status eco_step(eco_ctx* ctx, float lr, float beta1, float beta2, float eps,
                 break;
             case KIND_ROW:
                 ECO_CUDA(ctx, eco::launch_row(ctx->lc, descs, units, L.n_units, P, stream));
+                break;
+            case KIND_ROW_STREAM:
+                ECO_CUDA(ctx, eco::launch_stream(ctx->lc, eco::STREAM_ROW, descs, units, L.n_units, P, nullptr, nullptr,
+                                                 nullptr, false, ctx->d_tickets, ctx->d_status, ctx->grid_cap, stream));
                 break;
             case KIND_TENSOR:
                 ECO_CUDA(ctx, eco::launch_tensor_amax(ctx->lc, descs, units, L.n_units, P, ctx->d_amax[parity], ctx->d_s_old, stream));

@@ -21,8 +21,9 @@ int rows_per_unit();
 int stream_unit_rows();
 
 // Modes of the TMA-fed streaming kernel (eco_stream_kernels.cu).
-enum : int { STREAM_BLOCK = 0, STREAM_TENSOR_AMAX = 1, STREAM_TENSOR_APPLY = 2 };
-enum : int { MODE_BLOCK = STREAM_BLOCK, MODE_TENSOR_AMAX = STREAM_TENSOR_AMAX, MODE_TENSOR_APPLY = STREAM_TENSOR_APPLY };
+enum : int { STREAM_BLOCK = 0, STREAM_TENSOR_AMAX = 1, STREAM_TENSOR_APPLY = 2, STREAM_ROW = 3 };
+enum : int { MODE_BLOCK = STREAM_BLOCK, MODE_TENSOR_AMAX = STREAM_TENSOR_AMAX, MODE_TENSOR_APPLY = STREAM_TENSOR_APPLY,
+             MODE_ROW = STREAM_ROW };
 
 // Persistent launch over n_units work units; grid = min(n_units, grid_cap).  `tickets` are two device
 // words, zero before the first launch, that the kernel uses to hand out units and rewinds before it ends

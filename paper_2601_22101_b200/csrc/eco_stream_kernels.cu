@@ -40,8 +40,13 @@ struct StageHeader {
     uint32_t slot;
     float s_old;          // per-tensor modes
     float s_new, inv_new; // per-tensor pass 2
+    uint32_t seg_per_row; // per-row mode: 128-element rows per matrix row (R)
+    uint32_t div_magic;   // per-row mode: floor(65536 / R) + 1, so that (x * div_magic) >> 16 == x / R for x < 2048
+    uint32_t n_mrows;     // per-row mode: matrix rows in the unit
+    uint32_t pad_;
+    uint64_t mrow0;       // per-row mode: first matrix row of the unit
 };
-static_assert(sizeof(StageHeader) <= 64, "header must fit its slot");
+static_assert(sizeof(StageHeader) <= 128, "header must fit its slot");
 
 template <int FMT, int OPT>
 struct StageLayout {
@@ -54,7 +59,10 @@ struct StageLayout {
     static constexpr int kV = kM + kUnitRows * 512;
     static constexpr int kBytes = kV + (OPT == OPT_ADAM ? kUnitRows * 512 : 0);
     static constexpr int kStages = OPT == OPT_ADAM ? 2 : 3;
-    static constexpr int kBarriers = 128;                        // 2 * kStages mbarriers, padded
+    static constexpr int kBarriers = 512;                        // 2 * kStages + 2 mbarriers, padded to 128; then the
+                                                                 // per-row exchange: 32 maxima, 32 scales, 32 inverses
+    static constexpr int kRowBars = 64;                          // two mbarriers of the per-row exchange
+    static constexpr int kExchange = 128;
     static constexpr int kSmem = kBarriers + kStages * kBytes;
     static_assert(kBytes % 128 == 0, "stages stay 128-byte aligned");
 };
@@ -110,10 +118,11 @@ __device__ __forceinline__ uint32_t units_of(const TensorDesc& T) {
 // One unit (up to 32 rows of 128 elements) by the 8 consumer warps: warp w owns rows 4w..4w+3, lane l
 // elements 4l..4l+3 of each.  FULL: all 32 rows are present (every unit but the last of a tensor).
 template <int FMT, int OPT, int RND, int MODE, bool FULL>
-__device__ __forceinline__ void consume_unit(const StepParams& P, const int bf16_scale, const uint8_t* st,
+__device__ __forceinline__ bool consume_unit(const StepParams& P, const int bf16_scale, const uint8_t* st,
                                              const StageHeader* h, const uint32_t empty_bar, const int warp,
                                              const int lane, uint32_t* scratch_amax, uint32_t& cur_slot,
-                                             float& run_max) {
+                                             float& run_max, float* xchg, const uint32_t row_bars,
+                                             const uint32_t row_parity, uint32_t* status) {
     using SL = StageLayout<FMT, OPT>;
     const int r = warp * 4;
     const int nrows = FULL ? kUnitRows : static_cast<int>(h->nrows);
@@ -144,7 +153,9 @@ __device__ __forceinline__ void consume_unit(const StepParams& P, const int bf16
                     const float4 vr = *reinterpret_cast<const float4*>(st + SL::kV + row * 512 + lane * 16);
                     v[k][0] = vr.x; v[k][1] = vr.y; v[k][2] = vr.z; v[k][3] = vr.w;
                 }
-                s_old = MODE == MODE_BLOCK ? reinterpret_cast<const float*>(st + SL::kScales)[row] : h->s_old;
+                if (MODE == MODE_BLOCK) s_old = reinterpret_cast<const float*>(st + SL::kScales)[row];
+                else if (MODE == MODE_ROW) s_old = reinterpret_cast<const float*>(st + SL::kScales)[(row * h->div_magic) >> 16];
+                else s_old = h->s_old;
             }
             float val[4];
             unpack4<FMT>(codes, val);
@@ -168,6 +179,8 @@ __device__ __forceinline__ void consume_unit(const StepParams& P, const int bf16
     const uint64_t row0 = h->row0;
     const uint32_t tensor_id = h->tensor_id, slot = h->slot;
     const float s_new = h->s_new, inv_new = h->inv_new;
+    const uint32_t seg_per_row = h->seg_per_row, div_magic = h->div_magic, n_mrows = h->n_mrows;
+    const uint64_t mrow0 = h->mrow0;
     __syncwarp();
     if (lane == 0) mbar_arrive(empty_bar);          // the stage may be refilled
 
@@ -181,7 +194,7 @@ __device__ __forceinline__ void consume_unit(const StepParams& P, const int bf16
             run_max = 0.0f;
         }
         run_max = fmaxf(fmaxf(run_max, fmaxf(amax[0], amax[1])), fmaxf(amax[2], amax[3]));
-        return;
+        return true;
     }
 
     float s_k[4], inv_k[4];
@@ -203,6 +216,44 @@ __device__ __forceinline__ void consume_unit(const StepParams& P, const int bf16
             s_k[k] = __shfl_sync(0xFFFFFFFFu, s_mine, 8 * k);
             inv_k[k] = __shfl_sync(0xFFFFFFFFu, inv_mine, 8 * k);
         }
+    } else if (MODE == MODE_ROW) {
+        // One scale per matrix row = seg_per_row consecutive 128-element rows, which belong to several warps.
+        // Every warp posts the maxima of its 4 rows in shared memory; after the first barrier warp w reduces
+        // matrix rows w, w + 8, ... and posts scale and inverse; after the second barrier all read theirs.
+        // Both barriers are mbarriers with bounded waits (8 arrivals, one per consumer warp).
+        float* xmax = xchg;
+        float* xs = xchg + 32;
+        float* xinv = xchg + 64;
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            const float z = warp_amax(amax[k]);
+            if (lane == 0) xmax[r + k] = z;
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(row_bars);
+        if (!mbar_wait(row_bars, row_parity, status, 4u)) return false;
+        for (uint32_t j = static_cast<uint32_t>(warp); j < n_mrows; j += kConsumerWarps) {
+            const float x = static_cast<uint32_t>(lane) < seg_per_row ? xmax[j * seg_per_row + lane] : 0.0f;
+            const float a = warp_amax(x);
+            float s_j, inv_j;
+            uint32_t bits_j;
+            make_scale<FMT>(a, bf16_scale, s_j, inv_j, bits_j);
+            if (lane == 0) {
+                xs[j] = s_j;
+                xinv[j] = inv_j;
+                store_scale(sp, mrow0 + j, bf16_scale, s_j, bits_j);
+            }
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(row_bars + 8);
+        if (!mbar_wait(row_bars + 8, row_parity, status, 5u)) return false;
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            const uint32_t j = (static_cast<uint32_t>(r + k) * div_magic) >> 16;
+            const bool valid = FULL || r + k < nrows;
+            s_k[k] = valid ? xs[j] : 1.0f;
+            inv_k[k] = valid ? xinv[j] : 1.0f;
+        }
     } else {
 #pragma unroll
         for (int k = 0; k < 4; ++k) { s_k[k] = s_new; inv_k[k] = inv_new; }
@@ -222,12 +273,15 @@ __device__ __forceinline__ void consume_unit(const StepParams& P, const int bf16
         else *reinterpret_cast<uint16_t*>(wp + (i0 >> 1)) = static_cast<uint16_t>(codes);
         *reinterpret_cast<float4*>(mp + i0) = make_float4(mh[0], mh[1], mh[2], mh[3]);
     }
+    return true;
 }
 
 // ---------------------------------------------------------------------------
 // MODE_BLOCK        1x128 block scales, whole step in one pass
 // MODE_TENSOR_AMAX  per-tensor scale, pass 1: max |theta~| per tensor
 // MODE_TENSOR_APPLY per-tensor scale, pass 2: quantize with the tensor's scale
+// MODE_ROW          one scale per matrix row of up to 32 * 128 columns, whole step in one pass; a unit is
+//                   floor(32 / R) whole matrix rows of R 128-element rows each
 // Tensors handled here have a whole number of 128-element rows that start on
 // 128-element boundaries (cols % 128 == 0, or a flat tensor with numel % 128 == 0).
 // ---------------------------------------------------------------------------
@@ -244,6 +298,8 @@ eco_stream_kernel(const TensorDesc* __restrict__ descs, const uint32_t* __restri
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem);
     const uint32_t full0 = smem_addr(bars), empty0 = smem_addr(bars + S);
     uint8_t* stage0 = smem + SL::kBarriers;
+    const uint32_t row_bars = smem_addr(smem + SL::kRowBars);
+    float* xchg = reinterpret_cast<float*>(smem + SL::kExchange);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     if (threadIdx.x == 0) {
@@ -251,6 +307,8 @@ eco_stream_kernel(const TensorDesc* __restrict__ descs, const uint32_t* __restri
             mbar_init(full0 + 8 * s, 2);                 // producer: expect_tx arrival + header/scales arrival
             mbar_init(empty0 + 8 * s, kConsumerWarps);
         }
+        mbar_init(row_bars, kConsumerWarps);
+        mbar_init(row_bars + 8, kConsumerWarps);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
@@ -285,9 +343,13 @@ eco_stream_kernel(const TensorDesc* __restrict__ descs, const uint32_t* __restri
             if (!ok) break;
             uint8_t* st = stage0 + static_cast<size_t>(s) * SL::kBytes;
             const uint32_t local = unit - T.first_unit;
-            const uint64_t row0 = static_cast<uint64_t>(local) * kUnitRows;
+            const uint32_t unit_rows = MODE == MODE_ROW ? T.unit_rows : static_cast<uint32_t>(kUnitRows);
+            const uint64_t row0 = static_cast<uint64_t>(local) * unit_rows;
             const uint64_t left = T.n_blocks - row0;
-            const uint32_t nrows = left < kUnitRows ? static_cast<uint32_t>(left) : kUnitRows;
+            const uint32_t nrows = left < unit_rows ? static_cast<uint32_t>(left) : unit_rows;
+            const uint32_t mrows_per_unit = MODE == MODE_ROW ? unit_rows / T.blocks_per_row : 0u;
+            const uint64_t mrow0 = static_cast<uint64_t>(local) * mrows_per_unit;
+            const uint32_t n_mrows = MODE == MODE_ROW ? nrows / T.blocks_per_row : 0u;
             const uint32_t full = full0 + 8 * s;
             if (lane == 0) {
                 const uint32_t cb = nrows * SL::kCodeRow, gb = nrows * 256u, mb = nrows * 512u;
@@ -300,6 +362,8 @@ eco_stream_kernel(const TensorDesc* __restrict__ descs, const uint32_t* __restri
                 h.w = T.w; h.scale = T.scale; h.m = T.m; h.v = T.v;
                 h.row0 = row0; h.nrows = nrows; h.tensor_id = T.tensor_id; h.slot = T.slot;
                 h.s_old = 1.0f; h.s_new = 1.0f; h.inv_new = 1.0f;
+                h.seg_per_row = T.blocks_per_row; h.div_magic = 65536u / T.blocks_per_row + 1u;
+                h.n_mrows = n_mrows; h.pad_ = 0u; h.mrow0 = mrow0;
                 if (MODE == MODE_TENSOR_AMAX) {
                     h.s_old = load_scale(T.scale, 0, bf16_scale);
                     if (local == 0) scratch_s_old[T.slot] = h.s_old;
@@ -317,6 +381,8 @@ eco_stream_kernel(const TensorDesc* __restrict__ descs, const uint32_t* __restri
             }
             if (MODE == MODE_BLOCK && lane < static_cast<int>(nrows))
                 reinterpret_cast<float*>(st + SL::kScales)[lane] = load_scale(T.scale, row0 + lane, bf16_scale);
+            if (MODE == MODE_ROW && lane < static_cast<int>(n_mrows))
+                reinterpret_cast<float*>(st + SL::kScales)[lane] = load_scale(T.scale, mrow0 + lane, bf16_scale);
             __syncwarp();
             if (lane == 0) mbar_arrive(full);
             ++it;
@@ -358,10 +424,14 @@ eco_stream_kernel(const TensorDesc* __restrict__ descs, const uint32_t* __restri
         const uint32_t empty = empty0 + 8 * s;
         const uint32_t nrows = h->nrows;
         if (nrows == 0u) break;                   // end marker
+        bool ok;
         if (nrows == kUnitRows)
-            consume_unit<FMT, OPT, RND, MODE, true>(P, bf16_scale, st, h, empty, warp, lane, scratch_amax, cur_slot, run_max);
+            ok = consume_unit<FMT, OPT, RND, MODE, true>(P, bf16_scale, st, h, empty, warp, lane, scratch_amax, cur_slot,
+                                                         run_max, xchg, row_bars, it & 1u, status);
         else
-            consume_unit<FMT, OPT, RND, MODE, false>(P, bf16_scale, st, h, empty, warp, lane, scratch_amax, cur_slot, run_max);
+            ok = consume_unit<FMT, OPT, RND, MODE, false>(P, bf16_scale, st, h, empty, warp, lane, scratch_amax, cur_slot,
+                                                          run_max, xchg, row_bars, it & 1u, status);
+        if (!ok) return;
     }
     if (MODE == MODE_TENSOR_AMAX && cur_slot != 0xFFFFFFFFu) {
         const float z = warp_amax(run_max);
@@ -384,7 +454,8 @@ static cudaError_t launch_one(const TensorDesc* descs, const uint32_t* unit_tens
     }
     const uint32_t grid = n_units < static_cast<uint32_t>(grid_cap) ? n_units : static_cast<uint32_t>(grid_cap);
     kernel<<<grid, kStreamThreads, SL::kSmem, stream>>>(descs, unit_tensor, n_units, P, bf16_scale, amax, amax_next,
-                                                        s_old, reverse ? 1 : 0, MODE == MODE_BLOCK ? kInterleave : 1, tickets, status);
+                                                        s_old, reverse ? 1 : 0,
+                                                        (MODE == MODE_BLOCK || MODE == MODE_ROW) ? kInterleave : 1, tickets, status);
     return cudaGetLastError();
 }
 
@@ -409,6 +480,9 @@ cudaError_t launch_stream(const LaunchConfig& c, int mode, const TensorDesc* des
         }))
     }
     ECO_S_FMT(c.format, ECO_S_OPT(c.optimizer, ECO_S_RND(c.rounding, {
+        if (mode == STREAM_ROW)
+            return launch_one<F, O, R, MODE_ROW>(descs, unit_tensor, n_units, P, c.bf16_scale, amax, amax_next, s_old,
+                                                 reverse, tickets, status, grid_cap, stream);
         if (mode == STREAM_BLOCK)
             return launch_one<F, O, R, MODE_BLOCK>(descs, unit_tensor, n_units, P, c.bf16_scale, amax, amax_next, s_old,
                                                    reverse, tickets, status, grid_cap, stream);
