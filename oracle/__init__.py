@@ -91,6 +91,8 @@ def lib() -> ctypes.CDLL:
             getattr(L, f"eco_oracle_dequantize_{sfx}").argtypes = [vp, vp, vp, u64, u64, vp]
             getattr(L, f"eco_oracle_step_{sfx}").argtypes = [
                 vp, dbl, dbl, dbl, dbl, u64, u64, vp, vp, vp, vp, vp, u64, u64, u32, vp, vp, vp, vp]
+            getattr(L, f"eco_oracle_step_ex_{sfx}").argtypes = [
+                vp, dbl, dbl, dbl, dbl, dbl, dbl, u64, u64, vp, vp, vp, vp, vp, u64, u64, u32]
         _lib = L
     return _lib
 
@@ -166,9 +168,19 @@ def step(cfg: Config, *, lr: float, beta1: float, beta2: float = 0.0, eps: float
          step: int, seed: int = 0, w: np.ndarray, scale: np.ndarray | None, grad: np.ndarray,
          m: np.ndarray, v: np.ndarray | None = None, rows: int, cols: int, tensor_id: int = 0,
          noise: np.ndarray | None = None, e_prev: np.ndarray | None = None,
-         dbg_theta_tilde: np.ndarray | None = None, dbg_err: np.ndarray | None = None) -> None:
-    """One Algorithm-1 step on one tensor, in place.  ``m.dtype`` selects binary32 or binary64."""
+         dbg_theta_tilde: np.ndarray | None = None, dbg_err: np.ndarray | None = None,
+         weight_decay: float = 0.0, grad_scale: float = 1.0) -> None:
+    """One Algorithm-1 step on one tensor, in place.  ``m.dtype`` selects binary32 or binary64.
+    ``weight_decay`` (decoupled, AdamW style) and ``grad_scale`` (one factor on the gradient, e.g. the
+    clipping factor) are the two additions of Sec. 4's training recipe to OPTIM_STEP."""
     c = cfg.c()
+    if weight_decay != 0.0 or grad_scale != 1.0:
+        assert noise is None and e_prev is None and dbg_theta_tilde is None and dbg_err is None
+        rc = getattr(lib(), f"eco_oracle_step_ex_{_sfx(m.dtype)}")(
+            ctypes.byref(c), float(lr), float(beta1), float(beta2), float(eps), float(weight_decay), float(grad_scale),
+            int(step), int(seed), _ptr(w), _ptr(scale), _ptr(grad), _ptr(m), _ptr(v), rows, cols, tensor_id)
+        assert rc == 0
+        return
     rc = getattr(lib(), f"eco_oracle_step_{_sfx(m.dtype)}")(
         ctypes.byref(c), float(lr), float(beta1), float(beta2), float(eps), int(step), int(seed),
         _ptr(w), _ptr(scale), _ptr(grad), _ptr(m), _ptr(v), rows, cols, tensor_id,

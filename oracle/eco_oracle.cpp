@@ -316,6 +316,12 @@ struct Hyper {
     double lr, beta1, beta2, eps;
     uint64_t step;  // t, 1-based: the count of updates including this one
     uint64_t seed;
+    // The two ingredients every experiment of Sec. 4 adds to OPTIM_STEP ("AdamW ... weight decay of
+    // 0.1 and gradient clipping with a norm of 1.0") and that Algorithms 1-3 leave inside the optimizer's
+    // step function: decoupled weight decay lambda, and one global factor on the gradient (the clipping
+    // factor min(1, c / ||g||), computed by the caller).  0 and 1 switch them off.
+    double weight_decay = 0.0;
+    double grad_scale = 1.0;
 };
 
 template <class R>
@@ -323,6 +329,9 @@ struct StepScalars {
     R beta1, beta2, eps;
     R one_minus_beta1, one_minus_beta2;
     R neg_lr;          // SGDM: theta~ = theta^ - eta m~            (Eq. theta_tilde)
+    R neg_lr_wd;       // decoupled decay: theta^ <- theta^ - (eta lambda) theta^
+    R grad_scale;      // g <- grad_scale * g
+    bool decay;
     R alpha;           // SGDM: (1/eta)(1 - 1/beta)                 (Eq. alpha)
     R inv_lr;          // ideal injection (Appendix A): 1/eta
     R inv_lr_beta;     // ideal injection (Appendix A): 1/(eta beta)
@@ -343,6 +352,9 @@ StepScalars<R> derive_scalars(const Hyper& h) {
     s.one_minus_beta1 = R(1.0 - h.beta1);
     s.one_minus_beta2 = R(1.0 - h.beta2);
     s.neg_lr = R(-h.lr);
+    s.neg_lr_wd = R(-(h.lr * h.weight_decay));
+    s.grad_scale = R(h.grad_scale);
+    s.decay = h.weight_decay != 0.0;
     s.alpha = R((1.0 / h.lr) * (1.0 - 1.0 / h.beta1));
     s.inv_lr = R(1.0 / h.lr);
     s.inv_lr_beta = R(1.0 / (h.lr * h.beta1));
@@ -388,11 +400,13 @@ int step_tensor(const OracleConfig& cfg, const Hyper& hyper,
         R amax = R(0);
         for (uint64_t j = 0; j < len; ++j) {
             const uint64_t i = begin + j;
-            const R gi = cfg.grad_dtype == GRAD_BF16
-                             ? R(bf16_to_f32(static_cast<const uint16_t*>(grad)[i]))
-                             : static_cast<const R*>(grad)[i];
-            const R th = coded ? code_value<R>(cfg.format, load_code(cfg.format, static_cast<const uint8_t*>(w), i)) * s_old
-                               : static_cast<const R*>(w)[i];
+            const R graw = cfg.grad_dtype == GRAD_BF16
+                               ? R(bf16_to_f32(static_cast<const uint16_t*>(grad)[i]))
+                               : static_cast<const R*>(grad)[i];
+            const R gi = graw * sc.grad_scale;                                      // clipped / unscaled gradient
+            R th = coded ? code_value<R>(cfg.format, load_code(cfg.format, static_cast<const uint8_t*>(w), i)) * s_old
+                         : static_cast<const R*>(w)[i];
+            if (sc.decay) th = std::fma(sc.neg_lr_wd, th, th);                      // AdamW: theta (1 - eta lambda)
             R tht;
             const R mt = std::fma(sc.beta1, m[i], sc.one_minus_beta1 * gi);          // Eq. m_tilde
             if (cfg.optimizer == OPT_SGDM) {
@@ -502,6 +516,24 @@ int eco_oracle_step_f32(const OracleConfig* cfg, double lr, double beta1, double
     const Hyper h{lr, beta1, beta2, eps, step, seed};
     return step_tensor<float>(*cfg, h, w, scale, grad, m, v, rows, cols, tensor_id,
                               noise, e_prev, dbg_theta_tilde, dbg_err);
+}
+int eco_oracle_step_ex_f32(const OracleConfig* cfg, double lr, double beta1, double beta2, double eps,
+                           double weight_decay, double grad_scale, uint64_t step, uint64_t seed,
+                           void* w, void* scale, const void* grad, float* m, float* v,
+                           uint64_t rows, uint64_t cols, uint32_t tensor_id) {
+    Hyper h{lr, beta1, beta2, eps, step, seed};
+    h.weight_decay = weight_decay;
+    h.grad_scale = grad_scale;
+    return step_tensor<float>(*cfg, h, w, scale, grad, m, v, rows, cols, tensor_id, nullptr, nullptr, nullptr, nullptr);
+}
+int eco_oracle_step_ex_f64(const OracleConfig* cfg, double lr, double beta1, double beta2, double eps,
+                           double weight_decay, double grad_scale, uint64_t step, uint64_t seed,
+                           void* w, void* scale, const void* grad, double* m, double* v,
+                           uint64_t rows, uint64_t cols, uint32_t tensor_id) {
+    Hyper h{lr, beta1, beta2, eps, step, seed};
+    h.weight_decay = weight_decay;
+    h.grad_scale = grad_scale;
+    return step_tensor<double>(*cfg, h, w, scale, grad, m, v, rows, cols, tensor_id, nullptr, nullptr, nullptr, nullptr);
 }
 int eco_oracle_step_f64(const OracleConfig* cfg, double lr, double beta1, double beta2, double eps,
                         uint64_t step, uint64_t seed,

@@ -267,3 +267,64 @@ def test_memory_layout_matches_paper_count():
     w = wl.c4(layers=1, experts=2)
     assert w.state_bytes_per_param() == gold["state_bytes_per_param_fp8_adam_no_master"] == 9
     assert w.state_bytes_per_param() + (4 - 1) == gold["state_bytes_per_param_fp32_master"] == 12
+
+
+# --------------------------------------------------------------------------- Sec. 4 recipe: AdamW decay, clipping factor
+def test_identity_quantizer_with_decay_and_clipping_matches_adamw():
+    """Sec. 4.2 trains with AdamW (weight decay 0.1) and gradient clipping at norm 1.  With q = id the
+    step must be the library's AdamW on the clipped gradient: theta (1 - eta lambda) - eta_t m_hat."""
+    rng = np.random.default_rng(12)
+    n, lr, b1, b2, eps, wd, clip = 193, 2e-3, 0.9, 0.95, 1e-8, 0.1, 1.0
+    cfg = oracle.Config(format=IDENTITY, optimizer=ADAM, grad_dtype=GRAD_NATIVE)
+    theta0 = rng.standard_normal(n)
+    w, m, v = theta0.copy(), np.zeros(n), np.zeros(n)
+    p = torch.tensor(theta0, dtype=torch.float64, requires_grad=True)
+    topt = torch.optim.AdamW([p], lr=lr, betas=(b1, b2), eps=eps, weight_decay=wd)
+    for t in range(1, 16):
+        g = rng.standard_normal(n) * (3.0 if t % 2 else 0.01)          # clipped on odd steps, untouched on even ones
+        p.grad = torch.tensor(g)
+        total = float(torch.nn.utils.clip_grad_norm_([p], clip))
+        factor = min(1.0, clip / (total + 1e-6))                        # the factor torch applies
+        oracle.step(cfg, lr=lr, beta1=b1, beta2=b2, eps=eps, step=t, w=w, scale=None, grad=g, m=m, v=v,
+                    rows=1, cols=n, weight_decay=wd, grad_scale=factor)
+        topt.step()
+        np.testing.assert_allclose(w, p.detach().numpy(), rtol=1e-11, atol=1e-13)
+    np.testing.assert_allclose(m, topt.state[p]["exp_avg"].numpy(), rtol=1e-11, atol=1e-14)
+
+
+def test_sgdm_decoupled_decay_closed_form():
+    """One SGDM step with decay: theta~ = theta (1 - eta lambda) - eta (beta m + (1 - beta) c g)."""
+    cfg = oracle.Config(format=IDENTITY, optimizer=SGDM, grad_dtype=GRAD_NATIVE)
+    w, m, g = np.array([2.0, -1.0, 0.5]), np.array([0.1, 0.2, -0.3]), np.array([1.0, -2.0, 4.0])
+    lr, b, wd, c = 0.05, 0.8, 0.3, 0.25
+    expect_m = b * m + (1 - b) * (c * g)
+    expect_w = w * (1 - lr * wd) - lr * expect_m
+    oracle.step(cfg, lr=lr, beta1=b, step=1, w=w, scale=None, grad=g, m=m, rows=1, cols=3, weight_decay=wd, grad_scale=c)
+    np.testing.assert_allclose(w, expect_w, rtol=1e-14)
+    np.testing.assert_allclose(m, expect_m, rtol=1e-14)
+
+
+def test_grad_scale_equals_prescaled_gradient_bit_for_bit():
+    """A factor on the bf16 gradient is the same as handing in the binary32 product (quantized path, binary32)."""
+    rng = np.random.default_rng(13)
+    rows, cols, gs = 6, 256, 0.37
+    x = (rng.standard_normal((rows, cols)) * 0.02).astype(np.float32)
+    qcfg = oracle.Config(format=FP8_E4M3, granularity=PER_BLOCK, optimizer=ADAM, rounding=SR)
+    w0, s0 = oracle.quantize(oracle.Config(format=FP8_E4M3, granularity=PER_BLOCK), x)
+    g32 = (rng.standard_normal(rows * cols) * 1e-3).astype(np.float32)
+    gb = (g32.view(np.uint32) >> 16).astype(np.uint16)                  # bf16 patterns (truncation is fine here)
+    gf = (gb.astype(np.uint32) << 16).view(np.float32)
+    out = []
+    for variant in range(2):
+        w, s = w0.copy(), s0.copy()
+        m, v = np.zeros(rows * cols, np.float32), np.zeros(rows * cols, np.float32)
+        if variant == 0:
+            oracle.step(qcfg, lr=1e-3, beta1=0.9, beta2=0.95, eps=1e-8, step=1, seed=5, w=w, scale=s, grad=gb, m=m, v=v,
+                        rows=rows, cols=cols, grad_scale=gs)
+        else:
+            ncfg = oracle.Config(format=FP8_E4M3, granularity=PER_BLOCK, optimizer=ADAM, rounding=SR, grad_dtype=GRAD_NATIVE)
+            oracle.step(ncfg, lr=1e-3, beta1=0.9, beta2=0.95, eps=1e-8, step=1, seed=5, w=w, scale=s,
+                        grad=(gf * np.float32(gs)).astype(np.float32), m=m, v=v, rows=rows, cols=cols)
+        out.append((w, s, m, v))
+    for a, b in zip(out[0], out[1]):
+        assert (a.view(np.uint8) == b.view(np.uint8)).all()
