@@ -128,6 +128,27 @@ eco_status eco_step(eco_ctx* ctx, float lr, float beta1, float beta2, float eps,
                     uint64_t step, uint64_t seed, void* cuda_stream);
 
 /*
+ * eco_step_ex -- eco_step with the two additions the paper's training recipe makes to OPTIM_STEP
+ * (Sec. 4.2: AdamW with weight decay 0.1, gradient clipping at norm 1; Algorithms 1-3 leave both
+ * inside the optimizer's step function):
+ *   grad_scale    every gradient element is multiplied by this factor first (the clipping factor
+ *                 min(1, c / ||g||), or 1 / loss-scale; the caller computes it).  1 = off.
+ *   weight_decay  decoupled decay lambda: theta^ <- theta^ - (lr lambda) theta^ before the update,
+ *                 for SGDM and Adam alike.  0 = off.
+ * The error injection is unchanged.  With grad_scale = 1 and weight_decay = 0 the call is eco_step.
+ * Errors: as eco_step, plus ECO_ERR_INVALID_ARG for a NULL or non-zero-reserved struct, a negative
+ * or non-finite weight_decay, or a non-finite grad_scale.
+ */
+typedef struct eco_hyper {
+    float lr, beta1, beta2, eps;
+    float weight_decay, grad_scale;
+    uint64_t step; /* 1-based */
+    uint64_t seed;
+    uint64_t reserved; /* must be 0 */
+} eco_hyper;
+eco_status eco_step_ex(eco_ctx* ctx, const eco_hyper* hyper, void* cuda_stream);
+
+/*
  * eco_host_create / eco_host_step / eco_host_destroy -- the step of eco_step (Algorithm 1) for callers
  * that keep the state in HOST memory (offloaded optimizer state).  `tensors` has the layout of
  * eco_tensor but every pointer is a host pointer that must stay valid until eco_host_destroy (pinned

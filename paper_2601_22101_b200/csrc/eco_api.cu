@@ -169,7 +169,7 @@ eco_status check_hyper(eco_ctx* ctx, const eco_config& cfg, float lr, float beta
 
 // Scalars of one step, each derived in binary64 from the binary32 arguments and cast once.
 StepParams derive_params(const eco_config& cfg, float lr_f, float beta1_f, float beta2_f, float eps_f,
-                         uint64_t step, uint64_t seed) {
+                         uint64_t step, uint64_t seed, float weight_decay_f = 0.0f, float grad_scale_f = 1.0f) {
     const double lr = lr_f, b1 = beta1_f, b2 = beta2_f;
     const double t = static_cast<double>(step);
     StepParams P;
@@ -180,6 +180,10 @@ StepParams derive_params(const eco_config& cfg, float lr_f, float beta1_f, float
     P.one_minus_beta1 = static_cast<float>(1.0 - b1);
     P.one_minus_beta2 = static_cast<float>(1.0 - b2);
     P.neg_lr = -lr_f;
+    P.neg_lr_wd = static_cast<float>(-(lr * static_cast<double>(weight_decay_f)));
+    P.grad_scale = grad_scale_f;
+    P.has_decay = weight_decay_f != 0.0f ? 1 : 0;
+    P.has_grad_scale = grad_scale_f != 1.0f ? 1 : 0;
     P.alpha = static_cast<float>((1.0 / lr) * (1.0 - 1.0 / b1));
     if (cfg.optimizer == ECO_OPT_ADAM) {
         const double bc1 = 1.0 - std::pow(b1, t);
@@ -413,11 +417,38 @@ eco_status eco_create(eco_ctx** out, const eco_config* cfg, const eco_tensor* te
     return ECO_OK;
 }
 
+}  // extern "C"
+
+namespace {
+eco_status enqueue_step(eco_ctx* ctx, const StepParams& P, void* cuda_stream);
+}
+
+extern "C" {
+
 eco_status eco_step(eco_ctx* ctx, float lr, float beta1, float beta2, float eps,
                     uint64_t step, uint64_t seed, void* cuda_stream) {
     if (!ctx) return fail(nullptr, ECO_ERR_INVALID_ARG, "ctx is NULL");
     if (eco_status st = check_hyper(ctx, ctx->cfg, lr, beta1, beta2, eps, step)) return st;
-    const StepParams P = derive_params(ctx->cfg, lr, beta1, beta2, eps, step, seed);
+    return enqueue_step(ctx, derive_params(ctx->cfg, lr, beta1, beta2, eps, step, seed), cuda_stream);
+}
+
+eco_status eco_step_ex(eco_ctx* ctx, const eco_hyper* h, void* cuda_stream) {
+    if (!ctx) return fail(nullptr, ECO_ERR_INVALID_ARG, "ctx is NULL");
+    if (!h) return fail(ctx, ECO_ERR_INVALID_ARG, "hyper is NULL");
+    if (h->reserved != 0) return fail(ctx, ECO_ERR_INVALID_ARG, "hyper->reserved must be 0");
+    if (eco_status st = check_hyper(ctx, ctx->cfg, h->lr, h->beta1, h->beta2, h->eps, h->step)) return st;
+    if (!(h->weight_decay >= 0.0f) || !std::isfinite(h->weight_decay))
+        return fail(ctx, ECO_ERR_INVALID_ARG, "weight_decay must be finite and >= 0 (got %g)", h->weight_decay);
+    if (!std::isfinite(h->grad_scale)) return fail(ctx, ECO_ERR_INVALID_ARG, "grad_scale must be finite (got %g)", h->grad_scale);
+    return enqueue_step(ctx, derive_params(ctx->cfg, h->lr, h->beta1, h->beta2, h->eps, h->step, h->seed,
+                                           h->weight_decay, h->grad_scale), cuda_stream);
+}
+
+}  // extern "C"
+
+namespace {
+
+eco_status enqueue_step(eco_ctx* ctx, const StepParams& P, void* cuda_stream) {
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     const int parity = static_cast<int>(ctx->calls & 1);
     for (const Launch& L : ctx->launches) {
@@ -456,6 +487,10 @@ eco_status eco_step(eco_ctx* ctx, float lr, float beta1, float beta2, float eps,
     ctx->calls++;
     return ECO_OK;
 }
+
+}  // namespace
+
+extern "C" {
 
 eco_status eco_check(eco_ctx* ctx, void* cuda_stream) {
     if (!ctx) return fail(nullptr, ECO_ERR_INVALID_ARG, "ctx is NULL");

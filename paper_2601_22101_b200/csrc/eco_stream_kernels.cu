@@ -286,6 +286,8 @@ __device__ __forceinline__ bool consume_unit(const StepParams& P, const int bf16
 // 128-element boundaries (cols % 128 == 0, or a flat tensor with numel % 128 == 0).
 // ---------------------------------------------------------------------------
 template <int FMT, int OPT, int RND, int MODE>
+// Two CTAs per SM: the compiler then allows 96 registers per thread.  (112 would still add up to less than the
+// register file, but the hardware was measured to place only one such CTA per SM.)
 __global__ void __launch_bounds__(kStreamThreads, 2)
 eco_stream_kernel(const TensorDesc* __restrict__ descs, const uint32_t* __restrict__ unit_tensor,
                   const uint32_t n_units, const StepParams P, const int bf16_scale,

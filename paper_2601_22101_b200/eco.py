@@ -24,7 +24,7 @@ ECO_OPT_SGDM, ECO_OPT_ADAM = 0, 1
 ECO_ROUND_NEAREST, ECO_ROUND_STOCHASTIC = 0, 1
 ECO_INJECT_NONE, ECO_INJECT_ECO = 0, 1
 
-EXPORTED = ("eco_create", "eco_step", "eco_step_host", "eco_host_create", "eco_host_step", "eco_host_destroy",
+EXPORTED = ("eco_create", "eco_step", "eco_step_ex", "eco_step_host", "eco_host_create", "eco_host_step", "eco_host_destroy",
             "eco_step_static", "eco_check", "eco_destroy", "eco_last_error", "eco_quantize",
             "eco_set_option", "eco_num_launches", "eco_version")
 
@@ -38,6 +38,12 @@ class EcoError(RuntimeError):
 class eco_config(ctypes.Structure):
     _fields_ = [(n, ctypes.c_int32) for n in ("format", "granularity", "block", "scale_dtype", "optimizer",
                                               "rounding", "injection", "reserved")]
+
+
+class eco_hyper(ctypes.Structure):
+    _fields_ = [("lr", ctypes.c_float), ("beta1", ctypes.c_float), ("beta2", ctypes.c_float), ("eps", ctypes.c_float),
+                ("weight_decay", ctypes.c_float), ("grad_scale", ctypes.c_float),
+                ("step", ctypes.c_uint64), ("seed", ctypes.c_uint64), ("reserved", ctypes.c_uint64)]
 
 
 class eco_tensor(ctypes.Structure):
@@ -64,6 +70,8 @@ def load_library() -> ctypes.CDLL:
                                  ctypes.c_size_t, ctypes.c_int]
         L.eco_step.restype = ctypes.c_int
         L.eco_step.argtypes = [vp, f32, f32, f32, f32, u64, u64, vp]
+        L.eco_step_ex.restype = ctypes.c_int
+        L.eco_step_ex.argtypes = [vp, ctypes.POINTER(eco_hyper), vp]
         L.eco_step_host.restype = ctypes.c_int
         L.eco_step_host.argtypes = [ctypes.POINTER(eco_config), ctypes.POINTER(eco_tensor), ctypes.c_size_t,
                                     ctypes.c_int, f32, f32, f32, f32, u64, u64,
@@ -162,6 +170,15 @@ def eco_step(handle: int, lr: float, beta1: float, beta2: float, eps: float, ste
              stream: int = 0) -> None:
     """Enqueue one ECO step on ``stream`` (a raw cudaStream_t).  See ``eco_step`` in include/eco.h."""
     st = load_library().eco_step(handle, lr, beta1, beta2, eps, step, seed, stream)
+    if st != ECO_OK:
+        _raise(st, handle)
+
+
+def eco_step_ex(handle: int, lr: float, beta1: float, beta2: float, eps: float, step: int, seed: int,
+                weight_decay: float = 0.0, grad_scale: float = 1.0, stream: int = 0) -> None:
+    """eco_step with decoupled weight decay and a factor on the gradient.  See ``eco_step_ex`` in include/eco.h."""
+    h = eco_hyper(lr, beta1, beta2, eps, weight_decay, grad_scale, step, seed, 0)
+    st = load_library().eco_step_ex(handle, ctypes.byref(h), stream)
     if st != ECO_OK:
         _raise(st, handle)
 

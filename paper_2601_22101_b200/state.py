@@ -113,11 +113,14 @@ class DeviceState:
         self.handle = eco.eco_create(config_of(self.workload, injection), self.tensors, self.device)
         return self.handle
 
-    def step(self, step: int, stream: Optional[int] = None) -> None:
+    def step(self, step: int, stream: Optional[int] = None, weight_decay: float = 0.0, grad_scale: float = 1.0) -> None:
         w = self.workload
         if stream is None:
             stream = torch.cuda.current_stream().cuda_stream
-        eco.eco_step(self.handle, w.lr, w.beta1, w.beta2, w.eps, step, w.step_seed, stream)
+        if weight_decay != 0.0 or grad_scale != 1.0:
+            eco.eco_step_ex(self.handle, w.lr, w.beta1, w.beta2, w.eps, step, w.step_seed, weight_decay, grad_scale, stream)
+        else:
+            eco.eco_step(self.handle, w.lr, w.beta1, w.beta2, w.eps, step, w.step_seed, stream)
 
     def destroy(self) -> None:
         if self.handle is not None:

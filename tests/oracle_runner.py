@@ -36,7 +36,8 @@ class OracleState:
             self.m.append(np.zeros(t.numel, np.float32))
             self.v.append(np.zeros(t.numel, np.float32) if w.optimizer == wl.ADAM else None)
 
-    def step(self, step: int, grads: Optional[List[np.ndarray]] = None) -> None:
+    def step(self, step: int, grads: Optional[List[np.ndarray]] = None, weight_decay: float = 0.0,
+             grad_scale: float = 1.0) -> None:
         w = self.workload
 
         def one(i):
@@ -45,7 +46,8 @@ class OracleState:
             oracle.step(self.cfg, lr=float(np.float32(w.lr)), beta1=float(np.float32(w.beta1)),
                         beta2=float(np.float32(w.beta2)), eps=float(np.float32(w.eps)), step=step,
                         seed=w.step_seed, w=self.w[i], scale=self.scale[i], grad=g, m=self.m[i], v=self.v[i],
-                        rows=t.rows, cols=t.cols, tensor_id=t.tensor_id)
+                        rows=t.rows, cols=t.cols, tensor_id=t.tensor_id,
+                        weight_decay=float(np.float32(weight_decay)), grad_scale=float(np.float32(grad_scale)))
 
         order = sorted(range(len(w.tensors)), key=lambda i: -w.tensors[i].numel)
         if self.threads > 1 and len(order) > 1:

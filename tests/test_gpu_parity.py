@@ -40,7 +40,8 @@ def compare(dev: DeviceState, ora: OracleState, where=""):
             np.testing.assert_allclose(_np(d.v), ora.v[i], rtol=RTOL, atol=ATOL, err_msg=tag + " v")
 
 
-def run_chained(w: wl.Workload, steps: int, check_every: int = 1, injection=eco.ECO_INJECT_ECO):
+def run_chained(w: wl.Workload, steps: int, check_every: int = 1, injection=eco.ECO_INJECT_ECO, weight_decay=0.0,
+                grad_scale=1.0):
     dev = DeviceState(w)
     dev.init_from_host()
     ora = OracleState(w, injection=oracle.INJECT_ECO if injection == eco.ECO_INJECT_ECO else oracle.INJECT_NONE)
@@ -51,8 +52,8 @@ def run_chained(w: wl.Workload, steps: int, check_every: int = 1, injection=eco.
             grads = [wl.gradient_bf16(w, t, step) for t in w.tensors]
             for i, g in enumerate(grads):
                 dev.tensors[i].grad.view(torch.int16).copy_(torch.from_numpy(g.view(np.int16)))
-            dev.step(step)
-            ora.step(step, grads)
+            dev.step(step, weight_decay=weight_decay, grad_scale=grad_scale)
+            ora.step(step, grads, weight_decay=weight_decay, grad_scale=grad_scale)
             if step % check_every == 0 or step == steps:
                 torch.cuda.synchronize()
                 compare(dev, ora, f"step {step}")
@@ -138,6 +139,31 @@ def test_naive_removal_flag_matches_oracle():
     """Injection switched off (the naive regime of Sec. 3.4) on the same kernel."""
     w = _mini(wl.FP8_E4M3, wl.PER_BLOCK, wl.SCALE_F32, wl.SGDM, wl.SR, [(4, 512), (3, 200)])
     run_chained(w, steps=4, injection=eco.ECO_INJECT_NONE)
+
+
+@pytest.mark.parametrize("fmt,sdt,opt,gran", [(wl.FP8_E4M3, wl.SCALE_F32, wl.ADAM, wl.PER_BLOCK),
+                                              (wl.FP8_E4M3, wl.SCALE_F32, wl.ADAM, wl.PER_TENSOR),
+                                              (wl.FP8_E4M3, wl.SCALE_F32, wl.ADAM, wl.PER_ROW),
+                                              (wl.INT4, wl.SCALE_BF16, wl.SGDM, wl.PER_BLOCK)])
+@pytest.mark.parametrize("wd,gs", [(0.1, 1.0), (0.0, 0.37), (0.1, 0.37)])
+def test_step_ex_weight_decay_and_grad_scale(fmt, sdt, opt, gran, wd, gs):
+    """eco_step_ex: AdamW-style decoupled decay and a clipping factor on the gradient (the recipe of Sec. 4.2)."""
+    shapes = RAGGED + (RAGGED_FP8_ONLY if fmt == wl.FP8_E4M3 else [])
+    run_chained(_mini(fmt, gran, sdt, opt, wl.SR, shapes), steps=4, weight_decay=wd, grad_scale=gs)
+
+
+def test_step_ex_rejects_bad_arguments():
+    w = _mini(wl.FP8_E4M3, wl.PER_BLOCK, wl.SCALE_F32, wl.ADAM, wl.SR, [(2, 256)])
+    dev = DeviceState(w)
+    dev.init_from_host()
+    dev.create()
+    try:
+        for kw in ({"weight_decay": -0.1}, {"weight_decay": float("inf")}, {"grad_scale": float("nan")}):
+            with pytest.raises(eco.EcoError) as e:
+                eco.eco_step_ex(dev.handle, 1e-3, 0.9, 0.95, 1e-8, 1, 0, **kw)
+            assert e.value.status == eco.ECO_ERR_INVALID_ARG
+    finally:
+        dev.destroy()
 
 
 def test_c2_decoder_100_chained_steps_full_size():
