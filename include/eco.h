@@ -219,6 +219,17 @@ eco_status eco_step_static(const eco_config* cfg, const eco_tensor* tensors, siz
  */
 eco_status eco_check(eco_ctx* ctx, void* cuda_stream);
 
+/*
+ * eco_selftest_wait -- exercise the bounded device-side wait without any fault: launches one warp that
+ * waits on a shared-memory barrier nothing will ever arrive on, with a limit of limit_cycles SM clock
+ * cycles (1..2e9) instead of the kernels' two seconds.  The wait must expire, record its code and let the
+ * kernel end normally; the call then returns what eco_check reports, i.e. ECO_ERR_TIMEOUT when the
+ * mechanism works (ECO_OK would mean the wait was not bounded-and-reported), and clears the status word
+ * again so that the context stays usable.  Synchronizes cuda_stream.  Must not overlap an eco_step of the
+ * same context.  Errors: ECO_ERR_INVALID_ARG, ECO_ERR_CUDA.
+ */
+eco_status eco_selftest_wait(eco_ctx* ctx, int64_t limit_cycles, void* cuda_stream);
+
 /* eco_destroy -- free the context's tables and scratch (synchronizes the device). NULL is allowed. */
 eco_status eco_destroy(eco_ctx* ctx);
 

@@ -499,8 +499,21 @@ eco_status eco_check(eco_ctx* ctx, void* cuda_stream) {
     ECO_CUDA(ctx, cudaMemcpy(&code, ctx->d_status, sizeof code, cudaMemcpyDeviceToHost));
     if (code != 0)
         return fail(ctx, ECO_ERR_TIMEOUT, "a bounded wait inside a kernel expired (code %u: 1 = producer waiting for a free "
-                    "stage, 2 = producer draining its copies, 3 = consumer waiting for data)", code);
+                    "stage, 2 = producer draining its copies, 3 = consumer waiting for data, 4/5 = per-row exchange, 7 = self-test)", code);
     return ECO_OK;
+}
+
+eco_status eco_selftest_wait(eco_ctx* ctx, int64_t limit_cycles, void* cuda_stream) {
+    if (!ctx) return fail(nullptr, ECO_ERR_INVALID_ARG, "ctx is NULL");
+    if (limit_cycles < 1 || limit_cycles > 2000000000LL)
+        return fail(ctx, ECO_ERR_INVALID_ARG, "limit_cycles must be in 1..2e9 (got %lld)", static_cast<long long>(limit_cycles));
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    ECO_CUDA(ctx, eco::launch_wait_selftest(ctx->d_status, limit_cycles, stream));
+    const eco_status st = eco_check(ctx, cuda_stream);
+    // the status word is sticky by design; the self-test owns it for the length of the call
+    ECO_CUDA(ctx, cudaMemsetAsync(ctx->d_status, 0, sizeof(uint32_t), stream));
+    ECO_CUDA(ctx, cudaStreamSynchronize(stream));
+    return st;
 }
 
 eco_status eco_destroy(eco_ctx* ctx) {

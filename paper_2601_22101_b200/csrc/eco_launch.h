@@ -33,6 +33,9 @@ cudaError_t launch_stream(const LaunchConfig& c, int mode, const TensorDesc* des
                           uint32_t n_units, const StepParams& P, uint32_t* amax, uint32_t* amax_next, float* s_old,
                           bool reverse, uint32_t* tickets, uint32_t* status, int grid_cap, cudaStream_t stream);
 
+// One warp waits, for at most limit_cycles, on a barrier nothing arrives on; then writes code 7 to *status.
+cudaError_t launch_wait_selftest(uint32_t* status, long long limit_cycles, cudaStream_t stream);
+
 cudaError_t launch_block128(const LaunchConfig& c, const TensorDesc* descs, const uint32_t* unit_tensor,
                             uint32_t n_units, bool generic, const StepParams& P, cudaStream_t stream);
 cudaError_t launch_tensor_amax(const LaunchConfig& c, const TensorDesc* descs, const uint32_t* unit_tensor,

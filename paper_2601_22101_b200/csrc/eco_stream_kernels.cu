@@ -86,11 +86,12 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
     return ok != 0;
 }
 // Bounded wait; on expiry records `code` and returns false.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, uint32_t* status, uint32_t code) {
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, uint32_t* status, uint32_t code,
+                                          long long limit_cycles = kWaitLimitCycles) {
     if (mbar_try_wait(bar, parity)) return true;
     const long long t0 = clock64();
     while (!mbar_try_wait(bar, parity)) {
-        if (clock64() - t0 > kWaitLimitCycles) {
+        if (clock64() - t0 > limit_cycles) {
             atomicExch(status, code);
             return false;
         }
@@ -492,6 +493,23 @@ cudaError_t launch_stream(const LaunchConfig& c, int mode, const TensorDesc* des
                                                       s_old, reverse, tickets, status, grid_cap, stream);
     })))
     return cudaErrorInvalidValue;
+}
+
+// Self-test of the bounded wait: one warp waits on an mbarrier that nothing ever arrives on.  The wait
+// must give up after limit_cycles, record its code and let the kernel end normally.
+__global__ void eco_wait_selftest_kernel(uint32_t* status, long long limit_cycles) {
+    __shared__ __align__(8) uint64_t bar;
+    if (threadIdx.x == 0) {
+        mbar_init(smem_addr(&bar), 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+    mbar_wait(smem_addr(&bar), 0, status, 7u, limit_cycles);
+}
+
+cudaError_t launch_wait_selftest(uint32_t* status, long long limit_cycles, cudaStream_t stream) {
+    eco_wait_selftest_kernel<<<1, 32, 0, stream>>>(status, limit_cycles);
+    return cudaGetLastError();
 }
 
 int stream_unit_rows() { return kUnitRows; }

@@ -25,7 +25,7 @@ ECO_ROUND_NEAREST, ECO_ROUND_STOCHASTIC = 0, 1
 ECO_INJECT_NONE, ECO_INJECT_ECO = 0, 1
 
 EXPORTED = ("eco_create", "eco_step", "eco_step_ex", "eco_step_host", "eco_host_create", "eco_host_step", "eco_host_destroy",
-            "eco_step_static", "eco_check", "eco_destroy", "eco_last_error", "eco_quantize",
+            "eco_step_static", "eco_check", "eco_selftest_wait", "eco_destroy", "eco_last_error", "eco_quantize",
             "eco_set_option", "eco_num_launches", "eco_version")
 
 
@@ -88,6 +88,8 @@ def load_library() -> ctypes.CDLL:
                                       ctypes.c_int, f32, f32, f32, f32, u64, u64, vp]
         L.eco_check.restype = ctypes.c_int
         L.eco_check.argtypes = [vp, vp]
+        L.eco_selftest_wait.restype = ctypes.c_int
+        L.eco_selftest_wait.argtypes = [vp, i64, vp]
         L.eco_destroy.restype = ctypes.c_int
         L.eco_destroy.argtypes = [vp]
         L.eco_last_error.restype = ctypes.c_char_p
@@ -241,6 +243,11 @@ def eco_check(handle: int, stream: int = 0) -> None:
     st = load_library().eco_check(handle, stream)
     if st != ECO_OK:
         _raise(st, handle)
+
+
+def eco_selftest_wait(handle: int, limit_cycles: int = 2_000_000, stream: int = 0) -> int:
+    """Run the bounded-wait self-test; returns the status (ECO_ERR_TIMEOUT when the mechanism works)."""
+    return load_library().eco_selftest_wait(handle, limit_cycles, stream)
 
 
 def eco_destroy(handle: int) -> None:

@@ -326,3 +326,26 @@ def test_c5_full_size_sampled_tensors():
     w = wl.c5()
     ids = {0, 1, 2} | {3 + i for i in _spread(len(w.tensors) - 3, 18)}   # the dense layer (rows of 10944 = 85*128 + 64) + experts
     _sampled_full_size(w, sorted(ids))
+
+
+def test_bounded_wait_expires_and_reports_without_hurting_the_context():
+    """Failure detection without a GPU fault: a wait that nothing satisfies runs out after its limit, the kernel
+    ends normally, the host reads ECO_ERR_TIMEOUT, and the same context then steps correctly."""
+    w = _mini(wl.FP8_E4M3, wl.PER_BLOCK, wl.SCALE_F32, wl.ADAM, wl.SR, [(64, 512)])
+    dev = DeviceState(w)
+    dev.init_from_host()
+    ora = OracleState(w)
+    dev.create()
+    try:
+        stream = torch.cuda.current_stream().cuda_stream
+        assert eco.eco_selftest_wait(dev.handle, 2_000_000, stream) == eco.ECO_ERR_TIMEOUT
+        eco.eco_check(dev.handle, stream)                       # cleared again: no error
+        grads = [wl.gradient_bf16(w, t, 1) for t in w.tensors]
+        dev.tensors[0].grad.view(torch.int16).copy_(torch.from_numpy(grads[0].view(np.int16)))
+        dev.step(1)
+        ora.step(1, grads)
+        torch.cuda.synchronize()
+        compare(dev, ora, "after the self-test")
+        eco.eco_check(dev.handle, stream)
+    finally:
+        dev.destroy()
