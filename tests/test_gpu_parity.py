@@ -349,3 +349,18 @@ def test_bounded_wait_expires_and_reports_without_hurting_the_context():
         eco.eco_check(dev.handle, stream)
     finally:
         dev.destroy()
+
+
+def test_noise_floor_trends_of_sec_3_4_on_a_quadratic():
+    """Sec. 3.4 / Appendix C on a separable quadratic with the library's real FP8 quantizer (round to nearest):
+    as the learning rate shrinks the naive regime stalls ever farther from the optimum (floor growing roughly
+    like 1/eta), the ECO floor does not move and stays within a small factor of the master-weight floor."""
+    from paper_2601_22101_b200.examples.quadratic_floors import run
+    floors = {}
+    for lr, steps in ((0.3, 800), (0.03, 6000)):
+        for regime in ("master", "naive", "eco"):
+            floors[regime, lr] = run(regime, lr, steps, stochastic=False)
+    assert floors["naive", 0.03] > 10 * floors["naive", 0.3]            # naive: worse as eta shrinks
+    assert 0.6 < floors["eco", 0.03] / floors["eco", 0.3] < 1.6          # ECO: floor independent of eta
+    assert floors["eco", 0.03] < 2.0 * floors["master", 0.03]            # and close to the master-weight floor
+    assert floors["naive", 0.03] > 30 * floors["eco", 0.03]
