@@ -79,7 +79,10 @@ typedef struct eco_tensor {
     float* v;          /* in/out: second moment, f32 [rows*cols]; must be NULL for ECO_OPT_SGDM    */
     int64_t rows, cols;
     uint32_t tensor_id;/* selects the tensor's random stream; unique within a context              */
-    uint32_t reserved; /* must be 0                                                                */
+    uint32_t row_offset;/* 0 for a whole tensor.  For a shard made of rows [row_offset, row_offset + rows) of a
+                          larger tensor: the random stream is then drawn for the elements' positions in the
+                          whole tensor, so that shards round exactly like the unsplit tensor.  row_offset * cols
+                          must be a multiple of 4                                                          */
 } eco_tensor;
 
 /*
@@ -147,6 +150,26 @@ typedef struct eco_hyper {
     uint64_t reserved; /* must be 0 */
 } eco_hyper;
 eco_status eco_step_ex(eco_ctx* ctx, const eco_hyper* hyper, void* cuda_stream);
+
+/*
+ * eco_step_begin / eco_amax_buffer / eco_step_end -- eco_step_ex cut in two at the one point where a
+ * per-tensor scale needs the whole tensor (Sec. 3.1: s = max|x| / rho over everything that shares the
+ * scale), for tensors whose rows are split across several GPUs:
+ *   eco_step_begin   pass 1 on every tensor of the context: max |theta~| into the context's amax vector.
+ *   eco_amax_buffer  device pointer and length of that vector: n 32-bit words, entry i = bit pattern of the
+ *                    non-negative binary32 maximum of tensor i (bit patterns of non-negative floats order like
+ *                    unsigned integers).  Between begin and end the caller takes the element-wise MAXIMUM over
+ *                    the ranks that hold shards of the same tensors (one all-reduce with MAX on this vector, on
+ *                    the same stream), in place.  Every rank must list the same tensors in the same order.
+ *   eco_step_end     pass 2: derive each scale from the (reduced) maximum, quantize, inject, store.
+ * With row_offset set in the shards' eco_tensor entries the result is bit-identical to stepping the whole
+ * tensors in one context.  Only for ECO_SCALE_PER_TENSOR (other granularities shard with no exchange: use
+ * eco_step).  Errors: ECO_ERR_UNSUPPORTED for another granularity; ECO_ERR_INVALID_ARG for eco_step_end
+ * without a pending eco_step_begin, or eco_step / eco_step_begin while one is pending; otherwise as eco_step_ex.
+ */
+eco_status eco_step_begin(eco_ctx* ctx, const eco_hyper* hyper, void* cuda_stream);
+eco_status eco_amax_buffer(eco_ctx* ctx, void** device_ptr, size_t* n);
+eco_status eco_step_end(eco_ctx* ctx, void* cuda_stream);
 
 /*
  * eco_host_create / eco_host_step / eco_host_destroy -- the step of eco_step (Algorithm 1) for callers

@@ -55,6 +55,9 @@ struct eco_ctx {
     float* d_s_old = nullptr;
     uint32_t* d_status = nullptr;
     uint32_t* d_tickets = nullptr;
+    bool pending = false;          // eco_step_begin issued, eco_step_end not yet
+    StepParams pending_params{};
+    size_t n_tensors = 0;
     int grid_cap = 296;
     uint64_t calls = 0;
     bool reverse_pass2 = true;
@@ -251,7 +254,11 @@ eco_status eco_create(eco_ctx** out, const eco_config* cfg, const eco_tensor* te
     for (size_t i = 0; i < n; ++i) {
         const eco_tensor& t = tensors[i];
         if (eco_status st = check_shape(*cfg, t.rows, t.cols, i)) return st;
-        if (t.reserved != 0) return fail(nullptr, ECO_ERR_INVALID_ARG, "tensor %zu: reserved must be 0", i);
+        if ((static_cast<uint64_t>(t.row_offset) * static_cast<uint64_t>(t.cols)) % 4 != 0)
+            return fail(nullptr, ECO_ERR_INVALID_ARG, "tensor %zu: row_offset * cols must be a multiple of 4", i);
+        if (static_cast<unsigned __int128>(static_cast<uint64_t>(t.row_offset) + static_cast<uint64_t>(t.rows)) *
+                static_cast<unsigned __int128>(t.cols) >= (static_cast<unsigned __int128>(1) << 34))
+            return fail(nullptr, ECO_ERR_INVALID_ARG, "tensor %zu: (row_offset + rows) * cols must be < 2^34", i);
         if (!ids.insert(t.tensor_id).second) return fail(nullptr, ECO_ERR_INVALID_ARG, "tensor %zu: duplicate tensor_id %u", i, t.tensor_id);
         if (adam && !t.v) return fail(nullptr, ECO_ERR_INVALID_ARG, "tensor %zu: Adam needs v", i);
         if (!adam && t.v) return fail(nullptr, ECO_ERR_INVALID_ARG, "tensor %zu: v must be NULL for SGDM", i);
@@ -275,6 +282,7 @@ eco_status eco_create(eco_ctx** out, const eco_config* cfg, const eco_tensor* te
     if (!ctx) return fail(nullptr, ECO_ERR_NOMEM, "out of host memory");
     ctx->cfg = *cfg;
     ctx->device = device;
+    ctx->n_tensors = n;
     ctx->lc = launch_config(*cfg);
     ctx->reverse_pass2 = g_options.reverse_pass2 != 0;
     ctx->grid_cap = static_cast<int>(g_options.ctas_per_sm) * prop.multiProcessorCount;
@@ -298,6 +306,7 @@ eco_status eco_create(eco_ctx** out, const eco_config* cfg, const eco_tensor* te
         d.blocks_per_row = static_cast<uint32_t>((t.cols + 127) / 128);
         d.tensor_id = t.tensor_id;
         d.slot = static_cast<uint32_t>(i);
+        d.index_base = static_cast<uint64_t>(t.row_offset) * static_cast<uint64_t>(t.cols);
         return d;
     };
     // Appends one launch over the tensors `members`; returns false if the grid would overflow.
@@ -420,7 +429,8 @@ eco_status eco_create(eco_ctx** out, const eco_config* cfg, const eco_tensor* te
 }  // extern "C"
 
 namespace {
-eco_status enqueue_step(eco_ctx* ctx, const StepParams& P, void* cuda_stream);
+enum { PASS_BOTH = 0, PASS_AMAX = 1, PASS_APPLY = 2 };
+eco_status enqueue_step(eco_ctx* ctx, const StepParams& P, void* cuda_stream, int pass = PASS_BOTH);
 }
 
 extern "C" {
@@ -444,11 +454,46 @@ eco_status eco_step_ex(eco_ctx* ctx, const eco_hyper* h, void* cuda_stream) {
                                            h->weight_decay, h->grad_scale), cuda_stream);
 }
 
+eco_status eco_step_begin(eco_ctx* ctx, const eco_hyper* h, void* cuda_stream) {
+    if (!ctx) return fail(nullptr, ECO_ERR_INVALID_ARG, "ctx is NULL");
+    if (ctx->cfg.granularity != ECO_SCALE_PER_TENSOR)
+        return fail(ctx, ECO_ERR_UNSUPPORTED, "eco_step_begin / eco_step_end are for ECO_SCALE_PER_TENSOR; other granularities need no exchange");
+    if (!h) return fail(ctx, ECO_ERR_INVALID_ARG, "hyper is NULL");
+    if (h->reserved != 0) return fail(ctx, ECO_ERR_INVALID_ARG, "hyper->reserved must be 0");
+    if (eco_status st = check_hyper(ctx, ctx->cfg, h->lr, h->beta1, h->beta2, h->eps, h->step)) return st;
+    if (!(h->weight_decay >= 0.0f) || !std::isfinite(h->weight_decay))
+        return fail(ctx, ECO_ERR_INVALID_ARG, "weight_decay must be finite and >= 0 (got %g)", h->weight_decay);
+    if (!std::isfinite(h->grad_scale)) return fail(ctx, ECO_ERR_INVALID_ARG, "grad_scale must be finite (got %g)", h->grad_scale);
+    const StepParams P = derive_params(ctx->cfg, h->lr, h->beta1, h->beta2, h->eps, h->step, h->seed, h->weight_decay, h->grad_scale);
+    if (eco_status st = enqueue_step(ctx, P, cuda_stream, PASS_AMAX)) return st;
+    ctx->pending_params = P;
+    ctx->pending = true;
+    return ECO_OK;
+}
+
+eco_status eco_amax_buffer(eco_ctx* ctx, void** device_ptr, size_t* n) {
+    if (!ctx || !device_ptr || !n) return fail(ctx, ECO_ERR_INVALID_ARG, "NULL argument");
+    if (ctx->cfg.granularity != ECO_SCALE_PER_TENSOR) return fail(ctx, ECO_ERR_UNSUPPORTED, "only per-tensor scales have an amax vector");
+    *device_ptr = ctx->d_amax[ctx->calls & 1];
+    *n = ctx->n_tensors;
+    return ECO_OK;
+}
+
+eco_status eco_step_end(eco_ctx* ctx, void* cuda_stream) {
+    if (!ctx) return fail(nullptr, ECO_ERR_INVALID_ARG, "ctx is NULL");
+    if (!ctx->pending) return fail(ctx, ECO_ERR_INVALID_ARG, "eco_step_end without a pending eco_step_begin");
+    if (eco_status st = enqueue_step(ctx, ctx->pending_params, cuda_stream, PASS_APPLY)) return st;
+    ctx->pending = false;
+    return ECO_OK;
+}
+
 }  // extern "C"
 
 namespace {
 
-eco_status enqueue_step(eco_ctx* ctx, const StepParams& P, void* cuda_stream) {
+eco_status enqueue_step(eco_ctx* ctx, const StepParams& P, void* cuda_stream, int pass) {
+    if (ctx->pending && pass != PASS_APPLY)
+        return fail(ctx, ECO_ERR_INVALID_ARG, "eco_step_begin is pending: call eco_step_end first");
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     const int parity = static_cast<int>(ctx->calls & 1);
     for (const Launch& L : ctx->launches) {
@@ -463,12 +508,14 @@ eco_status enqueue_step(eco_ctx* ctx, const StepParams& P, void* cuda_stream) {
                 ECO_CUDA(ctx, eco::launch_block128(ctx->lc, descs, units, L.n_units, true, P, stream));
                 break;
             case KIND_TENSOR_STREAM:
-                ECO_CUDA(ctx, eco::launch_stream(ctx->lc, eco::STREAM_TENSOR_AMAX, descs, units, L.n_units, P,
-                                                 ctx->d_amax[parity], nullptr, ctx->d_s_old, false, ctx->d_tickets, ctx->d_status,
-                                                 ctx->grid_cap, stream));
-                ECO_CUDA(ctx, eco::launch_stream(ctx->lc, eco::STREAM_TENSOR_APPLY, descs, units, L.n_units, P,
-                                                 ctx->d_amax[parity], ctx->d_amax[parity ^ 1], ctx->d_s_old,
-                                                 ctx->reverse_pass2, ctx->d_tickets, ctx->d_status, ctx->grid_cap, stream));
+                if (pass != PASS_APPLY)
+                    ECO_CUDA(ctx, eco::launch_stream(ctx->lc, eco::STREAM_TENSOR_AMAX, descs, units, L.n_units, P,
+                                                     ctx->d_amax[parity], nullptr, ctx->d_s_old, false, ctx->d_tickets,
+                                                     ctx->d_status, ctx->grid_cap, stream));
+                if (pass != PASS_AMAX)
+                    ECO_CUDA(ctx, eco::launch_stream(ctx->lc, eco::STREAM_TENSOR_APPLY, descs, units, L.n_units, P,
+                                                     ctx->d_amax[parity], ctx->d_amax[parity ^ 1], ctx->d_s_old,
+                                                     ctx->reverse_pass2, ctx->d_tickets, ctx->d_status, ctx->grid_cap, stream));
                 break;
             case KIND_ROW:
                 ECO_CUDA(ctx, eco::launch_row(ctx->lc, descs, units, L.n_units, P, stream));
@@ -478,13 +525,15 @@ eco_status enqueue_step(eco_ctx* ctx, const StepParams& P, void* cuda_stream) {
                                                  nullptr, false, ctx->d_tickets, ctx->d_status, ctx->grid_cap, stream));
                 break;
             case KIND_TENSOR:
-                ECO_CUDA(ctx, eco::launch_tensor_amax(ctx->lc, descs, units, L.n_units, P, ctx->d_amax[parity], ctx->d_s_old, stream));
-                ECO_CUDA(ctx, eco::launch_tensor_apply(ctx->lc, descs, units, L.n_units, P, ctx->d_amax[parity],
-                                                       ctx->d_amax[parity ^ 1], ctx->d_s_old, ctx->reverse_pass2, stream));
+                if (pass != PASS_APPLY)
+                    ECO_CUDA(ctx, eco::launch_tensor_amax(ctx->lc, descs, units, L.n_units, P, ctx->d_amax[parity], ctx->d_s_old, stream));
+                if (pass != PASS_AMAX)
+                    ECO_CUDA(ctx, eco::launch_tensor_apply(ctx->lc, descs, units, L.n_units, P, ctx->d_amax[parity],
+                                                           ctx->d_amax[parity ^ 1], ctx->d_s_old, ctx->reverse_pass2, stream));
                 break;
         }
     }
-    ctx->calls++;
+    if (pass != PASS_AMAX) ctx->calls++;       // the amax slots alternate by step parity
     return ECO_OK;
 }
 
@@ -822,7 +871,8 @@ eco_status eco_step_static(const eco_config* cfg, const eco_tensor* tensors, siz
     for (size_t i = 0; i < n; ++i) {
         const eco_tensor& t = tensors[i];
         if (eco_status st = check_shape(*cfg, t.rows, t.cols, i)) return st;
-        if (t.reserved != 0) return fail(nullptr, ECO_ERR_INVALID_ARG, "tensor %zu: reserved must be 0", i);
+        if ((static_cast<uint64_t>(t.row_offset) * static_cast<uint64_t>(t.cols)) % 4 != 0)
+            return fail(nullptr, ECO_ERR_INVALID_ARG, "tensor %zu: row_offset * cols must be a multiple of 4", i);
         if (adam != (t.v != nullptr)) return fail(nullptr, ECO_ERR_INVALID_ARG, "tensor %zu: v must be given for Adam and NULL for SGDM", i);
         for (size_t j = 0; j < i; ++j)
             if (tensors[j].tensor_id == t.tensor_id) return fail(nullptr, ECO_ERR_INVALID_ARG, "tensor %zu: duplicate tensor_id %u", i, t.tensor_id);
@@ -845,6 +895,7 @@ eco_status eco_step_static(const eco_config* cfg, const eco_tensor* tensors, siz
         d.n_blocks = (d.numel + 127) / 128;
         d.tensor_id = t.tensor_id;
         d.slot = static_cast<uint32_t>(i);
+        d.index_base = static_cast<uint64_t>(t.row_offset) * static_cast<uint64_t>(t.cols);
         const uint64_t nu = (d.n_blocks + rpu - 1) / rpu;
         total += d.numel;
         if (units + nu > kStaticMaxUnits)

@@ -45,6 +45,7 @@ struct StageHeader {
     uint32_t n_mrows;     // per-row mode: matrix rows in the unit
     uint32_t pad_;
     uint64_t mrow0;       // per-row mode: first matrix row of the unit
+    uint64_t index_base;  // element index of the tensor's first element inside the full (unsharded) tensor
 };
 static_assert(sizeof(StageHeader) <= 128, "header must fit its slot");
 
@@ -181,7 +182,7 @@ __device__ __forceinline__ bool consume_unit(const StepParams& P, const int bf16
     const uint32_t tensor_id = h->tensor_id, slot = h->slot;
     const float s_new = h->s_new, inv_new = h->inv_new;
     const uint32_t seg_per_row = h->seg_per_row, div_magic = h->div_magic, n_mrows = h->n_mrows;
-    const uint64_t mrow0 = h->mrow0;
+    const uint64_t mrow0 = h->mrow0, index_base = h->index_base;
     __syncwarp();
     if (lane == 0) mbar_arrive(empty_bar);          // the stage may be refilled
 
@@ -265,7 +266,7 @@ __device__ __forceinline__ bool consume_unit(const StepParams& P, const int bf16
         const uint64_t i0 = i_first + k * 128;
         uint32_t word[4] = {0u, 0u, 0u, 0u};
         if (RND == RND_SR) {
-            const uint4 rw = philox4x32_10(static_cast<uint32_t>(i0 >> 2), tensor_id, P.step_lo, P.step_hi, P);
+            const uint4 rw = philox4x32_10(static_cast<uint32_t>((i0 + index_base) >> 2), tensor_id, P.step_lo, P.step_hi, P);
             word[0] = rw.x; word[1] = rw.y; word[2] = rw.z; word[3] = rw.w;
         }
         float mh[4];
@@ -366,7 +367,7 @@ eco_stream_kernel(const TensorDesc* __restrict__ descs, const uint32_t* __restri
                 h.row0 = row0; h.nrows = nrows; h.tensor_id = T.tensor_id; h.slot = T.slot;
                 h.s_old = 1.0f; h.s_new = 1.0f; h.inv_new = 1.0f;
                 h.seg_per_row = T.blocks_per_row; h.div_magic = 65536u / T.blocks_per_row + 1u;
-                h.n_mrows = n_mrows; h.pad_ = 0u; h.mrow0 = mrow0;
+                h.n_mrows = n_mrows; h.pad_ = 0u; h.mrow0 = mrow0; h.index_base = T.index_base;
                 if (MODE == MODE_TENSOR_AMAX) {
                     h.s_old = load_scale(T.scale, 0, bf16_scale);
                     if (local == 0) scratch_s_old[T.slot] = h.s_old;

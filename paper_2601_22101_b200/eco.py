@@ -24,7 +24,7 @@ ECO_OPT_SGDM, ECO_OPT_ADAM = 0, 1
 ECO_ROUND_NEAREST, ECO_ROUND_STOCHASTIC = 0, 1
 ECO_INJECT_NONE, ECO_INJECT_ECO = 0, 1
 
-EXPORTED = ("eco_create", "eco_step", "eco_step_ex", "eco_step_host", "eco_host_create", "eco_host_step", "eco_host_destroy",
+EXPORTED = ("eco_create", "eco_step", "eco_step_ex", "eco_step_begin", "eco_amax_buffer", "eco_step_end", "eco_step_host", "eco_host_create", "eco_host_step", "eco_host_destroy",
             "eco_step_static", "eco_check", "eco_selftest_wait", "eco_destroy", "eco_last_error", "eco_quantize",
             "eco_set_option", "eco_num_launches", "eco_version")
 
@@ -50,7 +50,7 @@ class eco_tensor(ctypes.Structure):
     _fields_ = [("w", ctypes.c_void_p), ("scale", ctypes.c_void_p), ("grad", ctypes.c_void_p),
                 ("m", ctypes.c_void_p), ("v", ctypes.c_void_p),
                 ("rows", ctypes.c_int64), ("cols", ctypes.c_int64),
-                ("tensor_id", ctypes.c_uint32), ("reserved", ctypes.c_uint32)]
+                ("tensor_id", ctypes.c_uint32), ("row_offset", ctypes.c_uint32)]
 
 
 _lib = None
@@ -72,6 +72,12 @@ def load_library() -> ctypes.CDLL:
         L.eco_step.argtypes = [vp, f32, f32, f32, f32, u64, u64, vp]
         L.eco_step_ex.restype = ctypes.c_int
         L.eco_step_ex.argtypes = [vp, ctypes.POINTER(eco_hyper), vp]
+        L.eco_step_begin.restype = ctypes.c_int
+        L.eco_step_begin.argtypes = [vp, ctypes.POINTER(eco_hyper), vp]
+        L.eco_amax_buffer.restype = ctypes.c_int
+        L.eco_amax_buffer.argtypes = [vp, ctypes.POINTER(vp), ctypes.POINTER(ctypes.c_size_t)]
+        L.eco_step_end.restype = ctypes.c_int
+        L.eco_step_end.argtypes = [vp, vp]
         L.eco_step_host.restype = ctypes.c_int
         L.eco_step_host.argtypes = [ctypes.POINTER(eco_config), ctypes.POINTER(eco_tensor), ctypes.c_size_t,
                                     ctypes.c_int, f32, f32, f32, f32, u64, u64,
@@ -132,6 +138,7 @@ class Tensor:
     rows: int
     cols: int
     tensor_id: int
+    row_offset: int = 0
 
 
 def _addr(x) -> Optional[int]:
@@ -152,7 +159,7 @@ def _tensor_array(tensors: Sequence[Tensor]):
     arr = (eco_tensor * len(tensors))()
     for i, t in enumerate(tensors):
         arr[i] = eco_tensor(_addr(t.w), _addr(t.scale), _addr(t.grad), _addr(t.m), _addr(t.v),
-                            t.rows, t.cols, t.tensor_id, 0)
+                            t.rows, t.cols, t.tensor_id, t.row_offset)
     return arr
 
 
@@ -183,6 +190,54 @@ def eco_step_ex(handle: int, lr: float, beta1: float, beta2: float, eps: float, 
     st = load_library().eco_step_ex(handle, ctypes.byref(h), stream)
     if st != ECO_OK:
         _raise(st, handle)
+
+
+def eco_step_begin(handle: int, lr: float, beta1: float, beta2: float, eps: float, step: int, seed: int,
+                   weight_decay: float = 0.0, grad_scale: float = 1.0, stream: int = 0) -> None:
+    """Pass 1 of a per-tensor-scale step (max|theta~| per tensor).  See ``eco_step_begin`` in include/eco.h."""
+    h = eco_hyper(lr, beta1, beta2, eps, weight_decay, grad_scale, step, seed, 0)
+    st = load_library().eco_step_begin(handle, ctypes.byref(h), stream)
+    if st != ECO_OK:
+        _raise(st, handle)
+
+
+class _DeviceWords:
+    """A view of n 32-bit words of device memory that torch can wrap without copying."""
+
+    def __init__(self, ptr: int, n: int):
+        self.__cuda_array_interface__ = {"shape": (n,), "typestr": "<i4", "data": (ptr, False), "version": 2}
+
+
+def eco_amax_tensor(handle: int, device: int = 0):
+    """The context's amax vector as a torch int32 CUDA tensor aliasing the library's memory (bit patterns of
+    non-negative floats: their integer order is their float order).  Reduce it with MAX across ranks in place
+    between ``eco_step_begin`` and ``eco_step_end``."""
+    import torch
+    ptr, n = ctypes.c_void_p(), ctypes.c_size_t()
+    st = load_library().eco_amax_buffer(handle, ctypes.byref(ptr), ctypes.byref(n))
+    if st != ECO_OK:
+        _raise(st, handle)
+    return torch.as_tensor(_DeviceWords(ptr.value, n.value), device=torch.device("cuda", device))
+
+
+def eco_step_end(handle: int, stream: int = 0) -> None:
+    """Pass 2 of a per-tensor-scale step.  See ``eco_step_end`` in include/eco.h."""
+    st = load_library().eco_step_end(handle, stream)
+    if st != ECO_OK:
+        _raise(st, handle)
+
+
+def eco_step_sharded(handle: int, lr: float, beta1: float, beta2: float, eps: float, step: int, seed: int,
+                     weight_decay: float = 0.0, grad_scale: float = 1.0, group=None, device: int = 0) -> None:
+    """One per-tensor-scale step of a context that holds ROW SHARDS of tensors whose other rows live on other
+    ranks of ``group`` (torch.distributed, NCCL): pass 1, one all-reduce(MAX) of the amax vector, pass 2.
+    Argument marshalling and one collective only; runs on the current torch stream."""
+    import torch
+    import torch.distributed as dist
+    stream = torch.cuda.current_stream(device).cuda_stream
+    eco_step_begin(handle, lr, beta1, beta2, eps, step, seed, weight_decay, grad_scale, stream)
+    dist.all_reduce(eco_amax_tensor(handle, device), op=dist.ReduceOp.MAX, group=group)
+    eco_step_end(handle, stream)
 
 
 def eco_step_host(cfg: Config, tensors: Sequence[Tensor], lr: float, beta1: float, beta2: float, eps: float,

@@ -364,3 +364,63 @@ def test_noise_floor_trends_of_sec_3_4_on_a_quadratic():
     assert 0.6 < floors["eco", 0.03] / floors["eco", 0.3] < 1.6          # ECO: floor independent of eta
     assert floors["eco", 0.03] < 2.0 * floors["master", 0.03]            # and close to the master-weight floor
     assert floors["naive", 0.03] > 30 * floors["eco", 0.03]
+
+
+@pytest.mark.parametrize("fmt,opt", [(wl.FP8_E4M3, wl.ADAM), (wl.INT4, wl.SGDM)])
+def test_row_shards_with_amax_exchange_equal_the_unsplit_step(fmt, opt):
+    """Per-tensor scales with tensors split by rows across ranks (emulated here as two contexts on one GPU, run
+    one after the other: no kernel waits on another): pass 1 on each shard, element-wise maximum of the two amax
+    vectors (what an all-reduce with MAX does), pass 2 on each shard.  With row_offset set the shards must hold
+    exactly the bits of the unsplit step: same scale, same stochastic rounding per element."""
+    shapes = [(64, 1024), (33, 384), (8, 640), (6, 200)]
+    w = _mini(fmt, wl.PER_TENSOR, wl.SCALE_F32, opt, wl.SR, shapes)
+    full = DeviceState(w)
+    full.init_from_host()
+    full.create()
+    adam = opt == wl.ADAM
+    shards = []          # per rank: (tensors, handle)
+    cuts = [t.rows // 2 for t in w.tensors]
+    per_row = lambda t: t.cols if fmt == wl.FP8_E4M3 else t.cols // 2
+    for rank in range(2):
+        ts = []
+        for i, (spec, d) in enumerate(zip(w.tensors, full.tensors)):
+            r0, r1 = (0, cuts[i]) if rank == 0 else (cuts[i], spec.rows)
+            sl = slice(r0 * spec.cols, r1 * spec.cols)
+            ts.append(eco.Tensor(d.w[r0 * per_row(spec): r1 * per_row(spec)].clone(), d.scale.clone(),
+                                 torch.zeros((r1 - r0) * spec.cols, dtype=torch.bfloat16, device="cuda"), d.m[sl].clone(),
+                                 d.v[sl].clone() if adam else None, r1 - r0, spec.cols, spec.tensor_id, row_offset=r0))
+        shards.append((ts, eco.eco_create(config_of(w), ts)))
+    stream = torch.cuda.current_stream().cuda_stream
+    try:
+        for step in (1, 2):
+            full.set_grads_from_host(step)
+            for rank, (ts, _) in enumerate(shards):
+                for i, (spec, d) in enumerate(zip(w.tensors, full.tensors)):
+                    r0, r1 = (0, cuts[i]) if rank == 0 else (cuts[i], spec.rows)
+                    ts[i].grad.copy_(d.grad[r0 * spec.cols: r1 * spec.cols])
+            full.step(step, weight_decay=0.05)
+            for _, h in shards:
+                eco.eco_step_begin(h, w.lr, w.beta1, w.beta2, w.eps, step, w.step_seed, 0.05, 1.0, stream)
+            a0, a1 = eco.eco_amax_tensor(shards[0][1]), eco.eco_amax_tensor(shards[1][1])
+            assert a0.numel() == len(shapes) and (a0 >= 0).all() and (a1 >= 0).all()
+            reduced = torch.maximum(a0, a1)
+            a0.copy_(reduced)
+            a1.copy_(reduced)
+            with pytest.raises(eco.EcoError):                    # a plain step while one is pending is refused
+                eco.eco_step(shards[0][1], w.lr, w.beta1, w.beta2, w.eps, step, w.step_seed, stream)
+            for _, h in shards:
+                eco.eco_step_end(h, stream)
+            torch.cuda.synchronize()
+            for i, (spec, d) in enumerate(zip(w.tensors, full.tensors)):
+                a, b = shards[0][0][i], shards[1][0][i]
+                assert torch.equal(torch.cat([a.w, b.w]), d.w), f"step {step} tensor {i}: codes"
+                assert torch.equal(a.scale.view(torch.int32), d.scale.view(torch.int32)) and torch.equal(a.scale, b.scale)
+                assert torch.equal(torch.cat([a.m, b.m]), d.m), f"step {step} tensor {i}: m"
+                if adam:
+                    assert torch.equal(torch.cat([a.v, b.v]), d.v)
+        with pytest.raises(eco.EcoError):
+            eco.eco_step_end(shards[0][1], stream)                # nothing pending
+    finally:
+        for _, h in shards:
+            eco.eco_destroy(h)
+        full.destroy()

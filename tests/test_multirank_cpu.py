@@ -68,6 +68,13 @@ def _worker(rank: int, world: int, port: int, q):
                 assert (cw == full.w[i]).all() and (cs.view(np.int32) == full.scale[i].view(np.int32)).all()
                 assert (cm.view(np.int32) == full.m[i].view(np.int32)).all()
                 assert (cv.view(np.int32) == full.v[i].view(np.int32)).all()
+        # the amax exchange of a row-sharded per-tensor step: an integer MAX over the bit patterns of
+        # non-negative binary32 values is their floating-point maximum
+        mine_amax = torch.tensor([0.0, 1e-30, 0.5 + rank, 3.0 - rank, 447.9999], dtype=torch.float32)
+        bits = mine_amax.view(torch.int32).clone()
+        dist.all_reduce(bits, op=dist.ReduceOp.MAX)
+        expect = torch.tensor([0.0, 1e-30, 0.5 + world - 1, 3.0, 447.9999], dtype=torch.float32)
+        assert torch.equal(bits.view(torch.float32), expect)
         # the benchmark's time reduction: max over ranks
         t = torch.tensor([10.0 + rank], dtype=torch.float64)
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
