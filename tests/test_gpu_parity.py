@@ -424,3 +424,12 @@ def test_row_shards_with_amax_exchange_equal_the_unsplit_step(fmt, opt):
         for _, h in shards:
             eco.eco_destroy(h)
         full.destroy()
+
+
+@pytest.mark.parametrize("fmt,sdt,opt", [(wl.FP8_E4M3, wl.SCALE_F32, wl.ADAM), (wl.INT4, wl.SCALE_BF16, wl.SGDM),
+                                         (wl.FP8_E4M3, wl.SCALE_BF16, wl.SGDM)])
+def test_per_row_scales_on_long_and_short_rows(fmt, sdt, opt):
+    """Per-row scales over the kernels that serve them: rows of up to 4096 columns made of whole 128-element
+    segments (streaming kernel, several matrix rows per unit), longer or ragged rows (one CTA per row)."""
+    shapes = [(5, 6912), (3, 12288), (2, 4224), (70, 1152), (9, 4096), (40, 128), (3, 8190), (4, 200)]
+    run_chained(_mini(fmt, wl.PER_ROW, sdt, opt, wl.SR, shapes), steps=5)
