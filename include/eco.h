@@ -56,7 +56,10 @@ enum { ECO_ROUND_NEAREST = 0,    /* ties to the even code                       
                                      seed, counter = (element index / 4, tensor_id, step), word = index mod 4;
                                      the top 24 bits of the word are compared with the fraction                  */
 enum { ECO_INJECT_NONE = 0, /* naive master-weight removal (Sec. 3.4): the error is dropped */
-       ECO_INJECT_ECO = 1 };/* the paper's method: m^ = m~ + alpha e                        */
+       ECO_INJECT_ECO = 1,  /* the paper's method: m^ = m~ + alpha e                        */
+       ECO_INJECT_EXACT = 2 };/* Appendix A: m <- m~ + e_t / eta - e_{t+1} / (eta beta) with the STORED error of the
+                               previous step; reproduces master-weight momentum SGD exactly, at the price of an FP32
+                               error buffer per parameter (eco_attach_error_buffers); momentum SGD only            */
 
 typedef struct eco_config {
     int32_t format;      /* ECO_FORMAT_*                                  */
@@ -241,6 +244,18 @@ eco_status eco_step_static(const eco_config* cfg, const eco_tensor* tensors, siz
  * Returns ECO_OK, ECO_ERR_TIMEOUT (state of the tensors is then undefined), or ECO_ERR_CUDA.
  */
 eco_status eco_check(eco_ctx* ctx, void* cuda_stream);
+
+/*
+ * eco_attach_error_buffers -- give every tensor of the context an FP32 buffer [rows*cols] (device,
+ * 16-byte aligned, zero before the first step) that each later step fills with the quantization error
+ * e_{t+1} = theta~_{t+1} - theta^_{t+1} of every element (Algorithm 2/3, line 2).  Two uses: ECO_INJECT_EXACT
+ * reads it back as e_t (Appendix A; without buffers such a context refuses to step), and with any injection
+ * it makes the error observable, e.g. for the consecutive-error statistics of Sec. 4.2 (Fig. 2).
+ *   e   host array of n device pointers, n = the context's tensor count, in the order of eco_create.
+ * Adds 4 bytes written (and, for ECO_INJECT_EXACT, 4 read) per parameter and step.  Synchronizes the device.
+ * Errors: ECO_ERR_INVALID_ARG, ECO_ERR_ALIGNMENT, ECO_ERR_CUDA.
+ */
+eco_status eco_attach_error_buffers(eco_ctx* ctx, float* const* e, size_t n);
 
 /*
  * eco_selftest_wait -- exercise the bounded device-side wait without any fault: launches one warp that

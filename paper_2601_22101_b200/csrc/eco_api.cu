@@ -56,6 +56,9 @@ struct eco_ctx {
     uint32_t* d_status = nullptr;
     uint32_t* d_tickets = nullptr;
     bool pending = false;          // eco_step_begin issued, eco_step_end not yet
+    std::vector<TensorDesc> h_descs;      // host copy of the descriptor table (patched by eco_attach_error_buffers)
+    std::vector<size_t> desc_of_tensor;   // tensor index -> its descriptor
+    bool has_error_buffers = false;
     StepParams pending_params{};
     size_t n_tensors = 0;
     int grid_cap = 296;
@@ -101,8 +104,10 @@ eco_status check_config(const eco_config* cfg, bool need_optimizer) {
     if (need_optimizer) {
         if (cfg->optimizer != ECO_OPT_SGDM && cfg->optimizer != ECO_OPT_ADAM)
             return fail(nullptr, ECO_ERR_UNSUPPORTED, "unknown optimizer %d", cfg->optimizer);
-        if (cfg->injection != ECO_INJECT_NONE && cfg->injection != ECO_INJECT_ECO)
+        if (cfg->injection != ECO_INJECT_NONE && cfg->injection != ECO_INJECT_ECO && cfg->injection != ECO_INJECT_EXACT)
             return fail(nullptr, ECO_ERR_UNSUPPORTED, "unknown injection %d", cfg->injection);
+        if (cfg->injection == ECO_INJECT_EXACT && cfg->optimizer != ECO_OPT_SGDM)
+            return fail(nullptr, ECO_ERR_UNSUPPORTED, "ECO_INJECT_EXACT (Appendix A) is defined for momentum SGD only");
     }
     if (cfg->reserved != 0) return fail(nullptr, ECO_ERR_INVALID_ARG, "cfg->reserved must be 0");
     return ECO_OK;
@@ -199,7 +204,9 @@ StepParams derive_params(const eco_config& cfg, float lr_f, float beta1_f, float
     P.seed_hi = static_cast<uint32_t>(seed >> 32);
     P.step_lo = static_cast<uint32_t>(step);
     P.step_hi = static_cast<uint32_t>(step >> 32);
-    P.inject = cfg.injection == ECO_INJECT_ECO ? 1 : 0;
+    P.inject = cfg.injection == ECO_INJECT_ECO ? 1 : (cfg.injection == ECO_INJECT_EXACT ? 2 : 0);
+    P.inv_lr = static_cast<float>(1.0 / lr);
+    P.inv_lr_beta = static_cast<float>(1.0 / (lr * b1));
     for (uint32_t r = 0; r < 10; ++r) {
         P.rk0[r] = P.seed_lo + r * 0x9E3779B9u;
         P.rk1[r] = P.seed_hi + r * 0xBB67AE85u;
@@ -288,6 +295,7 @@ eco_status eco_create(eco_ctx** out, const eco_config* cfg, const eco_tensor* te
     ctx->grid_cap = static_cast<int>(g_options.ctas_per_sm) * prop.multiProcessorCount;
     const bool use_stream = g_options.use_stream != 0;
 
+    ctx->desc_of_tensor.assign(n, 0);
     // ---- work-unit tables -------------------------------------------------
     const uint64_t rpu = static_cast<uint64_t>(eco::rows_per_unit());
     std::vector<TensorDesc> descs;
@@ -335,6 +343,7 @@ eco_status eco_create(eco_ctx** out, const eco_config* cfg, const eco_tensor* te
             }
             if (units + nu > 0x7FFFFFFFull) return false;
             d.first_unit = static_cast<uint32_t>(units);
+            ctx->desc_of_tensor[members[k]] = descs.size();
             descs.push_back(d);
             unit_tensor.insert(unit_tensor.end(), static_cast<size_t>(nu), static_cast<uint32_t>(k));
             units += nu;
@@ -408,6 +417,7 @@ eco_status eco_create(eco_ctx** out, const eco_config* cfg, const eco_tensor* te
     ECO_CUDA_CTX(cudaMalloc(&ctx->d_descs, descs.size() * sizeof(TensorDesc)));
     ECO_CUDA_CTX(cudaMalloc(&ctx->d_unit_tensor, std::max<size_t>(unit_tensor.size(), 1) * sizeof(uint32_t)));
     ECO_CUDA_CTX(cudaMemcpy(ctx->d_descs, descs.data(), descs.size() * sizeof(TensorDesc), cudaMemcpyHostToDevice));
+    ctx->h_descs = descs;
     ECO_CUDA_CTX(cudaMemcpy(ctx->d_unit_tensor, unit_tensor.data(), unit_tensor.size() * sizeof(uint32_t), cudaMemcpyHostToDevice));
     if (cfg->granularity == ECO_SCALE_PER_TENSOR) {
         for (int p = 0; p < 2; ++p) {
@@ -492,6 +502,8 @@ eco_status eco_step_end(eco_ctx* ctx, void* cuda_stream) {
 namespace {
 
 eco_status enqueue_step(eco_ctx* ctx, const StepParams& P, void* cuda_stream, int pass) {
+    if (P.inject == 2 && !ctx->has_error_buffers)
+        return fail(ctx, ECO_ERR_INVALID_ARG, "ECO_INJECT_EXACT needs eco_attach_error_buffers first");
     if (ctx->pending && pass != PASS_APPLY)
         return fail(ctx, ECO_ERR_INVALID_ARG, "eco_step_begin is pending: call eco_step_end first");
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
@@ -549,6 +561,20 @@ eco_status eco_check(eco_ctx* ctx, void* cuda_stream) {
     if (code != 0)
         return fail(ctx, ECO_ERR_TIMEOUT, "a bounded wait inside a kernel expired (code %u: 1 = producer waiting for a free "
                     "stage, 2 = producer draining its copies, 3 = consumer waiting for data, 4/5 = per-row exchange, 7 = self-test)", code);
+    return ECO_OK;
+}
+
+eco_status eco_attach_error_buffers(eco_ctx* ctx, float* const* e, size_t n) {
+    if (!ctx) return fail(nullptr, ECO_ERR_INVALID_ARG, "ctx is NULL");
+    if (!e || n != ctx->n_tensors) return fail(ctx, ECO_ERR_INVALID_ARG, "need one error buffer per tensor of the context (%zu)", ctx->n_tensors);
+    ECO_CUDA(ctx, cudaSetDevice(ctx->device));
+    for (size_t i = 0; i < n; ++i) {
+        if (eco_status st = check_device_ptr(e[i], ctx->device, "error buffer", i, true)) { ctx->err = g_thread_error; return st; }
+    }
+    for (size_t i = 0; i < n; ++i) ctx->h_descs[ctx->desc_of_tensor[i]].e = e[i];
+    ECO_CUDA(ctx, cudaDeviceSynchronize());
+    ECO_CUDA(ctx, cudaMemcpy(ctx->d_descs, ctx->h_descs.data(), ctx->h_descs.size() * sizeof(TensorDesc), cudaMemcpyHostToDevice));
+    ctx->has_error_buffers = true;
     return ECO_OK;
 }
 
@@ -859,6 +885,8 @@ eco_status eco_step_static(const eco_config* cfg, const eco_tensor* tensors, siz
     if (eco_status st = check_config(cfg, true)) return st;
     if (cfg->granularity != ECO_SCALE_PER_TENSOR)
         return fail(nullptr, ECO_ERR_UNSUPPORTED, "eco_step_static handles ECO_SCALE_PER_TENSOR only");
+    if (cfg->injection == ECO_INJECT_EXACT)
+        return fail(nullptr, ECO_ERR_UNSUPPORTED, "eco_step_static has no error buffers: ECO_INJECT_EXACT is not available");
     if (!tensors || n == 0) return fail(nullptr, ECO_ERR_INVALID_ARG, "empty tensor list");
     if (n > kStaticMaxTensors)
         return fail(nullptr, ECO_ERR_INVALID_ARG, "eco_step_static takes at most %u tensors per call (got %zu)",

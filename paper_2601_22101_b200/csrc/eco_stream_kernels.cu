@@ -46,6 +46,7 @@ struct StageHeader {
     uint32_t pad_;
     uint64_t mrow0;       // per-row mode: first matrix row of the unit
     uint64_t index_base;  // element index of the tensor's first element inside the full (unsharded) tensor
+    float* e;             // optional error buffer of the tensor (NULL: none)
 };
 static_assert(sizeof(StageHeader) <= 128, "header must fit its slot");
 
@@ -183,6 +184,7 @@ __device__ __forceinline__ bool consume_unit(const StepParams& P, const int bf16
     const float s_new = h->s_new, inv_new = h->inv_new;
     const uint32_t seg_per_row = h->seg_per_row, div_magic = h->div_magic, n_mrows = h->n_mrows;
     const uint64_t mrow0 = h->mrow0, index_base = h->index_base;
+    float* const ep = h->e;
     __syncwarp();
     if (lane == 0) mbar_arrive(empty_bar);          // the stage may be refilled
 
@@ -269,11 +271,16 @@ __device__ __forceinline__ bool consume_unit(const StepParams& P, const int bf16
             const uint4 rw = philox4x32_10(static_cast<uint32_t>((i0 + index_base) >> 2), tensor_id, P.step_lo, P.step_hi, P);
             word[0] = rw.x; word[1] = rw.y; word[2] = rw.z; word[3] = rw.w;
         }
-        float mh[4];
-        const uint32_t codes = back4<FMT, OPT, RND>(P, word, s_k[k], inv_k[k], L[k], mh);
+        float mh[4], e_prev[4] = {0.0f, 0.0f, 0.0f, 0.0f}, e_out[4];
+        if (ep && P.inject == 2) {
+            const float4 er = *reinterpret_cast<const float4*>(ep + i0);
+            e_prev[0] = er.x; e_prev[1] = er.y; e_prev[2] = er.z; e_prev[3] = er.w;
+        }
+        const uint32_t codes = back4<FMT, OPT, RND>(P, word, s_k[k], inv_k[k], L[k], mh, e_prev, e_out);
         if (FMT == FMT_FP8) *reinterpret_cast<uint32_t*>(wp + i0) = codes;
         else *reinterpret_cast<uint16_t*>(wp + (i0 >> 1)) = static_cast<uint16_t>(codes);
         *reinterpret_cast<float4*>(mp + i0) = make_float4(mh[0], mh[1], mh[2], mh[3]);
+        if (ep) *reinterpret_cast<float4*>(ep + i0) = make_float4(e_out[0], e_out[1], e_out[2], e_out[3]);
     }
     return true;
 }
@@ -367,7 +374,7 @@ eco_stream_kernel(const TensorDesc* __restrict__ descs, const uint32_t* __restri
                 h.row0 = row0; h.nrows = nrows; h.tensor_id = T.tensor_id; h.slot = T.slot;
                 h.s_old = 1.0f; h.s_new = 1.0f; h.inv_new = 1.0f;
                 h.seg_per_row = T.blocks_per_row; h.div_magic = 65536u / T.blocks_per_row + 1u;
-                h.n_mrows = n_mrows; h.pad_ = 0u; h.mrow0 = mrow0; h.index_base = T.index_base;
+                h.n_mrows = n_mrows; h.pad_ = 0u; h.mrow0 = mrow0; h.index_base = T.index_base; h.e = T.e;
                 if (MODE == MODE_TENSOR_AMAX) {
                     h.s_old = load_scale(T.scale, 0, bf16_scale);
                     if (local == 0) scratch_s_old[T.slot] = h.s_old;

@@ -22,10 +22,10 @@ ECO_SCALE_PER_TENSOR, ECO_SCALE_PER_ROW, ECO_SCALE_PER_BLOCK = 0, 1, 2
 ECO_SCALE_F32, ECO_SCALE_BF16 = 0, 1
 ECO_OPT_SGDM, ECO_OPT_ADAM = 0, 1
 ECO_ROUND_NEAREST, ECO_ROUND_STOCHASTIC = 0, 1
-ECO_INJECT_NONE, ECO_INJECT_ECO = 0, 1
+ECO_INJECT_NONE, ECO_INJECT_ECO, ECO_INJECT_EXACT = 0, 1, 2
 
 EXPORTED = ("eco_create", "eco_step", "eco_step_ex", "eco_step_begin", "eco_amax_buffer", "eco_step_end", "eco_step_host", "eco_host_create", "eco_host_step", "eco_host_destroy",
-            "eco_step_static", "eco_check", "eco_selftest_wait", "eco_destroy", "eco_last_error", "eco_quantize",
+            "eco_step_static", "eco_check", "eco_attach_error_buffers", "eco_selftest_wait", "eco_destroy", "eco_last_error", "eco_quantize",
             "eco_set_option", "eco_num_launches", "eco_version")
 
 
@@ -94,6 +94,8 @@ def load_library() -> ctypes.CDLL:
                                       ctypes.c_int, f32, f32, f32, f32, u64, u64, vp]
         L.eco_check.restype = ctypes.c_int
         L.eco_check.argtypes = [vp, vp]
+        L.eco_attach_error_buffers.restype = ctypes.c_int
+        L.eco_attach_error_buffers.argtypes = [vp, ctypes.POINTER(vp), ctypes.c_size_t]
         L.eco_selftest_wait.restype = ctypes.c_int
         L.eco_selftest_wait.argtypes = [vp, i64, vp]
         L.eco_destroy.restype = ctypes.c_int
@@ -296,6 +298,14 @@ def eco_step_static(cfg: Config, tensors: Sequence[Tensor], lr: float, beta1: fl
 def eco_check(handle: int, stream: int = 0) -> None:
     """Synchronize ``stream`` and raise if a bounded device-side wait expired.  See include/eco.h."""
     st = load_library().eco_check(handle, stream)
+    if st != ECO_OK:
+        _raise(st, handle)
+
+
+def eco_attach_error_buffers(handle: int, buffers) -> None:
+    """Attach one FP32 error buffer per tensor (torch CUDA tensors).  See ``eco_attach_error_buffers`` in include/eco.h."""
+    arr = (ctypes.c_void_p * len(buffers))(*[_addr(b) for b in buffers])
+    st = load_library().eco_attach_error_buffers(handle, arr, len(buffers))
     if st != ECO_OK:
         _raise(st, handle)
 

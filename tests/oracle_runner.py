@@ -35,6 +35,8 @@ class OracleState:
             self.scale.append(cs)
             self.m.append(np.zeros(t.numel, np.float32))
             self.v.append(np.zeros(t.numel, np.float32) if w.optimizer == wl.ADAM else None)
+        # the quantization error of the last step per tensor (read back by the exact injection of Appendix A)
+        self.e = [np.zeros(t.numel, np.float32) for t in w.tensors]
 
     def step(self, step: int, grads: Optional[List[np.ndarray]] = None, weight_decay: float = 0.0,
              grad_scale: float = 1.0) -> None:
@@ -43,6 +45,14 @@ class OracleState:
         def one(i):
             t = w.tensors[i]
             g = grads[i] if grads is not None else wl.gradient_bf16(w, t, step)
+            if weight_decay == 0.0 and grad_scale == 1.0:
+                ideal = self.cfg.injection == oracle.INJECT_IDEAL
+                err = None if ideal else self.e[i]
+                oracle.step(self.cfg, lr=float(np.float32(w.lr)), beta1=float(np.float32(w.beta1)),
+                            beta2=float(np.float32(w.beta2)), eps=float(np.float32(w.eps)), step=step,
+                            seed=w.step_seed, w=self.w[i], scale=self.scale[i], grad=g, m=self.m[i], v=self.v[i],
+                            rows=t.rows, cols=t.cols, tensor_id=t.tensor_id, e_prev=self.e[i] if ideal else None, dbg_err=err)
+                return
             oracle.step(self.cfg, lr=float(np.float32(w.lr)), beta1=float(np.float32(w.beta1)),
                         beta2=float(np.float32(w.beta2)), eps=float(np.float32(w.eps)), step=step,
                         seed=w.step_seed, w=self.w[i], scale=self.scale[i], grad=g, m=self.m[i], v=self.v[i],

@@ -355,11 +355,15 @@ def test_noise_floor_trends_of_sec_3_4_on_a_quadratic():
     """Sec. 3.4 / Appendix C on a separable quadratic with the library's real FP8 quantizer (round to nearest):
     as the learning rate shrinks the naive regime stalls ever farther from the optimum (floor growing roughly
     like 1/eta), the ECO floor does not move and stays within a small factor of the master-weight floor."""
-    from paper_2601_22101_b200.examples.quadratic_floors import run
+    from paper_2601_22101_b200.examples.quadratic_floors import error_similarity, run
     floors = {}
     for lr, steps in ((0.3, 800), (0.03, 6000)):
-        for regime in ("master", "naive", "eco"):
+        for regime in ("master", "naive", "eco", "exact"):
             floors[regime, lr] = run(regime, lr, steps, stochastic=False)
+        # Appendix A: with the stored error the run without master weights IS the master-weight run
+        assert abs(floors["exact", lr] / floors["master", lr] - 1.0) < 1e-3
+    ratio, cosine = error_similarity(0.03, 3000)                         # Sec. 3.2 / Fig. 2: e_{t+1} is close to e_t
+    assert 0.98 < ratio < 1.02 and cosine > 0.9
     assert floors["naive", 0.03] > 10 * floors["naive", 0.3]            # naive: worse as eta shrinks
     assert 0.6 < floors["eco", 0.03] / floors["eco", 0.3] < 1.6          # ECO: floor independent of eta
     assert floors["eco", 0.03] < 2.0 * floors["master", 0.03]            # and close to the master-weight floor
@@ -433,3 +437,35 @@ def test_per_row_scales_on_long_and_short_rows(fmt, sdt, opt):
     segments (streaming kernel, several matrix rows per unit), longer or ragged rows (one CTA per row)."""
     shapes = [(5, 6912), (3, 12288), (2, 4224), (70, 1152), (9, 4096), (40, 128), (3, 8190), (4, 200)]
     run_chained(_mini(fmt, wl.PER_ROW, sdt, opt, wl.SR, shapes), steps=5)
+
+
+@pytest.mark.parametrize("fmt,gran,rnd", [(wl.FP8_E4M3, wl.PER_BLOCK, wl.SR), (wl.FP8_E4M3, wl.PER_TENSOR, wl.RTN),
+                                          (wl.INT4, wl.PER_ROW, wl.SR)])
+@pytest.mark.parametrize("injection", [eco.ECO_INJECT_EXACT, eco.ECO_INJECT_ECO])
+def test_error_buffers_and_exact_injection(fmt, gran, rnd, injection):
+    """Attached error buffers receive e_{t+1} of every element at each step; ECO_INJECT_EXACT (Appendix A) reads them
+    back as e_t.  Both against the oracle, which pins the exact rule to master-weight momentum SGD on the CPU."""
+    shapes = RAGGED + (RAGGED_FP8_ONLY if fmt == wl.FP8_E4M3 else [])
+    w = _mini(fmt, gran, wl.SCALE_F32, wl.SGDM, rnd, shapes)
+    dev = DeviceState(w)
+    dev.init_from_host()
+    ora = OracleState(w, injection=oracle.INJECT_IDEAL if injection == eco.ECO_INJECT_EXACT else oracle.INJECT_ECO)
+    dev.create(injection)
+    ebufs = [torch.zeros(t.numel, dtype=torch.float32, device="cuda") for t in w.tensors]
+    try:
+        if injection == eco.ECO_INJECT_EXACT:
+            with pytest.raises(eco.EcoError):                      # refuses to step without its buffers
+                dev.step(1)
+        eco.eco_attach_error_buffers(dev.handle, ebufs)
+        for step in range(1, 6):
+            grads = [wl.gradient_bf16(w, t, step) for t in w.tensors]
+            for i, g in enumerate(grads):
+                dev.tensors[i].grad.view(torch.int16).copy_(torch.from_numpy(g.view(np.int16)))
+            dev.step(step)
+            ora.step(step, grads)
+            torch.cuda.synchronize()
+            compare(dev, ora, f"step {step}")
+            for i in range(len(w.tensors)):
+                assert (ebufs[i].cpu().numpy().view(np.int32) == ora.e[i].view(np.int32)).all(), f"step {step} tensor {i}: error buffer"
+    finally:
+        dev.destroy()
