@@ -514,7 +514,7 @@ eco_status enqueue_step(eco_ctx* ctx, const StepParams& P, void* cuda_stream, in
         switch (L.kind) {
             case KIND_BLOCK_FAST:
                 ECO_CUDA(ctx, eco::launch_stream(ctx->lc, eco::STREAM_BLOCK, descs, units, L.n_units, P, nullptr, nullptr,
-                                                 nullptr, false, ctx->d_tickets, ctx->d_status, ctx->grid_cap, stream));
+                                                 nullptr, false, ctx->d_tickets, ctx->d_status, ctx->grid_cap, stream, ctx->has_error_buffers));
                 break;
             case KIND_BLOCK_GENERIC:
                 ECO_CUDA(ctx, eco::launch_block128(ctx->lc, descs, units, L.n_units, true, P, stream));
@@ -527,14 +527,14 @@ eco_status enqueue_step(eco_ctx* ctx, const StepParams& P, void* cuda_stream, in
                 if (pass != PASS_AMAX)
                     ECO_CUDA(ctx, eco::launch_stream(ctx->lc, eco::STREAM_TENSOR_APPLY, descs, units, L.n_units, P,
                                                      ctx->d_amax[parity], ctx->d_amax[parity ^ 1], ctx->d_s_old,
-                                                     ctx->reverse_pass2, ctx->d_tickets, ctx->d_status, ctx->grid_cap, stream));
+                                                     ctx->reverse_pass2, ctx->d_tickets, ctx->d_status, ctx->grid_cap, stream, ctx->has_error_buffers));
                 break;
             case KIND_ROW:
                 ECO_CUDA(ctx, eco::launch_row(ctx->lc, descs, units, L.n_units, P, stream));
                 break;
             case KIND_ROW_STREAM:
                 ECO_CUDA(ctx, eco::launch_stream(ctx->lc, eco::STREAM_ROW, descs, units, L.n_units, P, nullptr, nullptr,
-                                                 nullptr, false, ctx->d_tickets, ctx->d_status, ctx->grid_cap, stream));
+                                                 nullptr, false, ctx->d_tickets, ctx->d_status, ctx->grid_cap, stream, ctx->has_error_buffers));
                 break;
             case KIND_TENSOR:
                 if (pass != PASS_APPLY)

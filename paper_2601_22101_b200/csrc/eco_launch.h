@@ -28,10 +28,12 @@ enum : int { MODE_BLOCK = STREAM_BLOCK, MODE_TENSOR_AMAX = STREAM_TENSOR_AMAX, M
 // Persistent launch over n_units work units; grid = min(n_units, grid_cap).  `tickets` are two device
 // words, zero before the first launch, that the kernel uses to hand out units and rewinds before it ends
 // (launches sharing them must be ordered on the device).  `status` is a device word that receives a
-// non-zero code if a bounded wait inside the kernel expires.
+// non-zero code if a bounded wait inside the kernel expires.  with_errors selects the instantiation that also
+// reads / writes the tensors' error buffers (TensorDesc::e must then be set for every tensor of the launch).
 cudaError_t launch_stream(const LaunchConfig& c, int mode, const TensorDesc* descs, const uint32_t* unit_tensor,
                           uint32_t n_units, const StepParams& P, uint32_t* amax, uint32_t* amax_next, float* s_old,
-                          bool reverse, uint32_t* tickets, uint32_t* status, int grid_cap, cudaStream_t stream);
+                          bool reverse, uint32_t* tickets, uint32_t* status, int grid_cap, cudaStream_t stream,
+                          bool with_errors = false);
 
 // One warp waits, for at most limit_cycles, on a barrier nothing arrives on; then writes code 7 to *status.
 cudaError_t launch_wait_selftest(uint32_t* status, long long limit_cycles, cudaStream_t stream);

@@ -120,7 +120,7 @@ __device__ __forceinline__ uint32_t units_of(const TensorDesc& T) {
 
 // One unit (up to 32 rows of 128 elements) by the 8 consumer warps: warp w owns rows 4w..4w+3, lane l
 // elements 4l..4l+3 of each.  FULL: all 32 rows are present (every unit but the last of a tensor).
-template <int FMT, int OPT, int RND, int MODE, bool FULL>
+template <int FMT, int OPT, int RND, int MODE, bool FULL, bool ERR>
 __device__ __forceinline__ bool consume_unit(const StepParams& P, const int bf16_scale, const uint8_t* st,
                                              const StageHeader* h, const uint32_t empty_bar, const int warp,
                                              const int lane, uint32_t* scratch_amax, uint32_t& cur_slot,
@@ -272,15 +272,15 @@ __device__ __forceinline__ bool consume_unit(const StepParams& P, const int bf16
             word[0] = rw.x; word[1] = rw.y; word[2] = rw.z; word[3] = rw.w;
         }
         float mh[4], e_prev[4] = {0.0f, 0.0f, 0.0f, 0.0f}, e_out[4];
-        if (ep && P.inject == 2) {
+        if (ERR && P.inject == 2) {
             const float4 er = *reinterpret_cast<const float4*>(ep + i0);
             e_prev[0] = er.x; e_prev[1] = er.y; e_prev[2] = er.z; e_prev[3] = er.w;
         }
-        const uint32_t codes = back4<FMT, OPT, RND>(P, word, s_k[k], inv_k[k], L[k], mh, e_prev, e_out);
+        const uint32_t codes = back4<FMT, OPT, RND, ERR>(P, word, s_k[k], inv_k[k], L[k], mh, e_prev, e_out);
         if (FMT == FMT_FP8) *reinterpret_cast<uint32_t*>(wp + i0) = codes;
         else *reinterpret_cast<uint16_t*>(wp + (i0 >> 1)) = static_cast<uint16_t>(codes);
         *reinterpret_cast<float4*>(mp + i0) = make_float4(mh[0], mh[1], mh[2], mh[3]);
-        if (ep) *reinterpret_cast<float4*>(ep + i0) = make_float4(e_out[0], e_out[1], e_out[2], e_out[3]);
+        if (ERR) *reinterpret_cast<float4*>(ep + i0) = make_float4(e_out[0], e_out[1], e_out[2], e_out[3]);
     }
     return true;
 }
@@ -294,7 +294,9 @@ __device__ __forceinline__ bool consume_unit(const StepParams& P, const int bf16
 // Tensors handled here have a whole number of 128-element rows that start on
 // 128-element boundaries (cols % 128 == 0, or a flat tensor with numel % 128 == 0).
 // ---------------------------------------------------------------------------
-template <int FMT, int OPT, int RND, int MODE>
+// ERR: the tensors carry error buffers (see eco_attach_error_buffers); a separate instantiation, so that the plain
+// method pays nothing for the option.
+template <int FMT, int OPT, int RND, int MODE, bool ERR>
 // Two CTAs per SM: the compiler then allows 96 registers per thread.  (112 would still add up to less than the
 // register file, but the hardware was measured to place only one such CTA per SM.)
 __global__ void __launch_bounds__(kStreamThreads, 2)
@@ -437,10 +439,10 @@ eco_stream_kernel(const TensorDesc* __restrict__ descs, const uint32_t* __restri
         if (nrows == 0u) break;                   // end marker
         bool ok;
         if (nrows == kUnitRows)
-            ok = consume_unit<FMT, OPT, RND, MODE, true>(P, bf16_scale, st, h, empty, warp, lane, scratch_amax, cur_slot,
+            ok = consume_unit<FMT, OPT, RND, MODE, true, ERR>(P, bf16_scale, st, h, empty, warp, lane, scratch_amax, cur_slot,
                                                          run_max, xchg, row_bars, it & 1u, status);
         else
-            ok = consume_unit<FMT, OPT, RND, MODE, false>(P, bf16_scale, st, h, empty, warp, lane, scratch_amax, cur_slot,
+            ok = consume_unit<FMT, OPT, RND, MODE, false, ERR>(P, bf16_scale, st, h, empty, warp, lane, scratch_amax, cur_slot,
                                                           run_max, xchg, row_bars, it & 1u, status);
         if (!ok) return;
     }
@@ -451,13 +453,13 @@ eco_stream_kernel(const TensorDesc* __restrict__ descs, const uint32_t* __restri
 }
 
 // ---------------------------------------------------------------------------
-template <int FMT, int OPT, int RND, int MODE>
+template <int FMT, int OPT, int RND, int MODE, bool ERR = false>
 static cudaError_t launch_one(const TensorDesc* descs, const uint32_t* unit_tensor, uint32_t n_units, const StepParams& P,
                               int bf16_scale, uint32_t* amax, uint32_t* amax_next, float* s_old, bool reverse,
                               uint32_t* tickets, uint32_t* status, int grid_cap, cudaStream_t stream) {
     using SL = StageLayout<FMT, OPT>;
     static bool configured = false;
-    auto kernel = eco_stream_kernel<FMT, OPT, RND, MODE>;
+    auto kernel = eco_stream_kernel<FMT, OPT, RND, MODE, ERR>;
     if (!configured) {
         cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SL::kSmem);
         if (e != cudaSuccess) return e;
@@ -482,7 +484,8 @@ static cudaError_t launch_one(const TensorDesc* descs, const uint32_t* unit_tens
 
 cudaError_t launch_stream(const LaunchConfig& c, int mode, const TensorDesc* descs, const uint32_t* unit_tensor,
                           uint32_t n_units, const StepParams& P, uint32_t* amax, uint32_t* amax_next, float* s_old,
-                          bool reverse, uint32_t* tickets, uint32_t* status, int grid_cap, cudaStream_t stream) {
+                          bool reverse, uint32_t* tickets, uint32_t* status, int grid_cap, cudaStream_t stream,
+                          bool with_errors) {
     if (n_units == 0) return cudaSuccess;
     if (mode == STREAM_TENSOR_AMAX) {
         ECO_S_FMT(c.format, ECO_S_OPT(c.optimizer, {
@@ -490,16 +493,20 @@ cudaError_t launch_stream(const LaunchConfig& c, int mode, const TensorDesc* des
                                                                amax_next, s_old, reverse, tickets, status, grid_cap, stream);
         }))
     }
+#define ECO_S_LAUNCH(MODE_, ERR_)                                                                                      \
+    return launch_one<F, O, R, MODE_, ERR_>(descs, unit_tensor, n_units, P, c.bf16_scale, amax, amax_next, s_old, reverse, \
+                                            tickets, status, grid_cap, stream)
     ECO_S_FMT(c.format, ECO_S_OPT(c.optimizer, ECO_S_RND(c.rounding, {
-        if (mode == STREAM_ROW)
-            return launch_one<F, O, R, MODE_ROW>(descs, unit_tensor, n_units, P, c.bf16_scale, amax, amax_next, s_old,
-                                                 reverse, tickets, status, grid_cap, stream);
-        if (mode == STREAM_BLOCK)
-            return launch_one<F, O, R, MODE_BLOCK>(descs, unit_tensor, n_units, P, c.bf16_scale, amax, amax_next, s_old,
-                                                   reverse, tickets, status, grid_cap, stream);
-        return launch_one<F, O, R, MODE_TENSOR_APPLY>(descs, unit_tensor, n_units, P, c.bf16_scale, amax, amax_next,
-                                                      s_old, reverse, tickets, status, grid_cap, stream);
+        if (with_errors) {
+            if (mode == STREAM_ROW) ECO_S_LAUNCH(MODE_ROW, true);
+            if (mode == STREAM_BLOCK) ECO_S_LAUNCH(MODE_BLOCK, true);
+            ECO_S_LAUNCH(MODE_TENSOR_APPLY, true);
+        }
+        if (mode == STREAM_ROW) ECO_S_LAUNCH(MODE_ROW, false);
+        if (mode == STREAM_BLOCK) ECO_S_LAUNCH(MODE_BLOCK, false);
+        ECO_S_LAUNCH(MODE_TENSOR_APPLY, false);
     })))
+#undef ECO_S_LAUNCH
     return cudaErrorInvalidValue;
 }
 
