@@ -293,6 +293,20 @@ eco_status eco_quantize(const eco_config* cfg, const float* x, int64_t rows, int
                         int device, void* cuda_stream);
 
 /*
+ * eco_dequantize -- x^ = value(code) * scale (Sec. 3.1, x^ = s y) for a whole tensor: the weights the
+ * forward and backward pass of quantized training read.  No master weights are involved: this only
+ * expands the stored codes.
+ *   w, scale  device, in: layouts as in eco_tensor (cfg gives format, granularity and scale dtype;
+ *             optimizer, rounding and injection are ignored).
+ *   out       device, out, 16-byte aligned: f32 [rows*cols], or bf16 [rows*cols] when out_bf16 != 0
+ *             (the product is then rounded to bf16, nearest even; INT4 values times a bf16 scale and
+ *             most FP8 products need the rounding).
+ * Asynchronous on cuda_stream.  Errors: as eco_quantize.
+ */
+eco_status eco_dequantize(const eco_config* cfg, const void* w, const void* scale, int64_t rows, int64_t cols,
+                          void* out, int out_bf16, int device, void* cuda_stream);
+
+/*
  * eco_set_option -- process-wide tuning knobs read by the NEXT eco_create:
  *   "l2_group_bytes"  per-tensor scales only: bytes of inputs one pass-1/pass-2 launch pair
  *                     covers (0, the default: one pair for the whole context, which measured

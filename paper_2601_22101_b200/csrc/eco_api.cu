@@ -817,6 +817,24 @@ eco_status eco_host_step(eco_host_ctx* h, float lr, float beta1, float beta2, fl
     return ECO_OK;
 }
 
+eco_status eco_dequantize(const eco_config* cfg, const void* w, const void* scale, int64_t rows, int64_t cols,
+                          void* out, int out_bf16, int device, void* cuda_stream) {
+    if (eco_status st = check_config(cfg, false)) return st;
+    if (eco_status st = check_shape(*cfg, rows, cols, 0)) return st;
+    ECO_CUDA(nullptr, cudaSetDevice(device));
+    if (eco_status st = check_device_ptr(w, device, "w", 0, true)) return st;
+    if (eco_status st = check_device_ptr(scale, device, "scale", 0, true)) return st;
+    if (eco_status st = check_device_ptr(out, device, "out", 0, true)) return st;
+    int sms = 148;
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device);
+    const uint64_t quads = static_cast<uint64_t>(rows) * static_cast<uint64_t>((cols + 3) / 4);
+    const uint32_t grid = static_cast<uint32_t>(std::max<uint64_t>(1, std::min<uint64_t>(static_cast<uint64_t>(sms) * 16, (quads + 255) / 256)));
+    ECO_CUDA(nullptr, eco::launch_dequantize(launch_config(*cfg), static_cast<const uint8_t*>(w), scale, out,
+                                             static_cast<uint64_t>(rows), static_cast<uint32_t>(cols), cfg->granularity,
+                                             out_bf16 != 0, grid, static_cast<cudaStream_t>(cuda_stream)));
+    return ECO_OK;
+}
+
 eco_status eco_step_host(const eco_config* cfg, const eco_tensor* tensors, size_t n, int device,
                          float lr, float beta1, float beta2, float eps, uint64_t step, uint64_t seed,
                          uint64_t* h2d_bytes, uint64_t* d2h_bytes) {

@@ -402,6 +402,47 @@ cudaError_t launch_quantize(const LaunchConfig& c, const float* x, uint8_t* w, v
     return cudaGetLastError();
 }
 
+// ---------------------------------------------------------------------------
+// x^ = value(code) * scale (Sec. 3.1) for a whole tensor: what the forward pass of quantized training reads.
+// One thread per 4 consecutive elements of a row (cols is even for INT4, so a thread never splits a byte);
+// gran: 0 per-tensor, 1 per-row, 2 blocks of 128 along the row.  OUT_BF16: round the product to bf16 (nearest even).
+// ---------------------------------------------------------------------------
+template <int FMT, bool OUT_BF16>
+__global__ void __launch_bounds__(kThreads)
+eco_dequantize_kernel(const uint8_t* __restrict__ w, const void* __restrict__ scale, void* __restrict__ out,
+                      const uint64_t rows, const uint32_t cols, const int gran, const int bf16_scale) {
+    const uint32_t quads_per_row = (cols + 3u) / 4u;
+    const uint64_t n_quads = rows * quads_per_row;
+    for (uint64_t qd = static_cast<uint64_t>(blockIdx.x) * kThreads + threadIdx.x; qd < n_quads;
+         qd += static_cast<uint64_t>(gridDim.x) * kThreads) {
+        const uint64_t row = qd / quads_per_row;
+        const uint32_t c0 = static_cast<uint32_t>(qd - row * quads_per_row) * 4u;
+        const int nvalid = static_cast<int>(min(4u, cols - c0));
+        const uint64_t i0 = row * cols + c0;
+        const bool vec = (i0 & 3) == 0;
+        const uint32_t codes = load_codes4<FMT>(w, i0, nvalid, vec);
+        float val[4];
+        unpack4<FMT>(codes, val);
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            if (e >= nvalid) break;
+            const uint64_t k = gran == 0 ? 0 : (gran == 1 ? row : row * ((cols + 127u) / 128u) + (c0 + e) / 128u);
+            const float x = __fmul_rn(val[e], load_scale(scale, k, bf16_scale));
+            if (OUT_BF16) static_cast<uint16_t*>(out)[i0 + e] = static_cast<uint16_t>(f32_to_bf16_bits_rne(x));
+            else static_cast<float*>(out)[i0 + e] = x;
+        }
+    }
+}
+
+cudaError_t launch_dequantize(const LaunchConfig& c, const uint8_t* w, const void* scale, void* out, uint64_t rows,
+                              uint32_t cols, int gran, bool out_bf16, uint32_t grid, cudaStream_t stream) {
+    ECO_DISPATCH_FMT(c.format, {
+        if (out_bf16) eco_dequantize_kernel<F, true><<<grid, kThreads, 0, stream>>>(w, scale, out, rows, cols, gran, c.bf16_scale);
+        else eco_dequantize_kernel<F, false><<<grid, kThreads, 0, stream>>>(w, scale, out, rows, cols, gran, c.bf16_scale);
+    })
+    return cudaGetLastError();
+}
+
 int rows_per_unit() { return kRowsPerUnit; }
 
 }  // namespace eco

@@ -53,4 +53,7 @@ cudaError_t launch_quantize(const LaunchConfig& c, const float* x, uint8_t* w, v
                             uint32_t cols, int mode, const StepParams& P, uint32_t tensor_id,
                             uint32_t* scratch_amax, uint32_t grid, cudaStream_t stream);
 
+cudaError_t launch_dequantize(const LaunchConfig& c, const uint8_t* w, const void* scale, void* out, uint64_t rows,
+                              uint32_t cols, int gran, bool out_bf16, uint32_t grid, cudaStream_t stream);
+
 }  // namespace eco

@@ -25,7 +25,7 @@ ECO_ROUND_NEAREST, ECO_ROUND_STOCHASTIC = 0, 1
 ECO_INJECT_NONE, ECO_INJECT_ECO, ECO_INJECT_EXACT = 0, 1, 2
 
 EXPORTED = ("eco_create", "eco_step", "eco_step_ex", "eco_step_begin", "eco_amax_buffer", "eco_step_end", "eco_step_host", "eco_host_create", "eco_host_step", "eco_host_destroy",
-            "eco_step_static", "eco_check", "eco_attach_error_buffers", "eco_selftest_wait", "eco_destroy", "eco_last_error", "eco_quantize",
+            "eco_step_static", "eco_check", "eco_attach_error_buffers", "eco_selftest_wait", "eco_destroy", "eco_last_error", "eco_quantize", "eco_dequantize",
             "eco_set_option", "eco_num_launches", "eco_version")
 
 
@@ -104,6 +104,8 @@ def load_library() -> ctypes.CDLL:
         L.eco_last_error.argtypes = [vp]
         L.eco_quantize.restype = ctypes.c_int
         L.eco_quantize.argtypes = [ctypes.POINTER(eco_config), vp, i64, i64, vp, vp, u64, u64, u32, ctypes.c_int, vp]
+        L.eco_dequantize.restype = ctypes.c_int
+        L.eco_dequantize.argtypes = [ctypes.POINTER(eco_config), vp, vp, i64, i64, vp, ctypes.c_int, ctypes.c_int, vp]
         L.eco_set_option.restype = ctypes.c_int
         L.eco_set_option.argtypes = [ctypes.c_char_p, i64]
         L.eco_num_launches.restype = ctypes.c_int
@@ -325,6 +327,16 @@ def eco_quantize(cfg: Config, x, rows: int, cols: int, w, scale, seed: int = 0, 
     c = cfg.c()
     st = load_library().eco_quantize(ctypes.byref(c), _addr(x), rows, cols, _addr(w), _addr(scale),
                                      seed, step, tensor_id, device, stream)
+    if st != ECO_OK:
+        _raise(st)
+
+
+def eco_dequantize(cfg: Config, w, scale, rows: int, cols: int, out, device: int = 0, stream: int = 0) -> None:
+    """out = value(code) * scale; ``out`` is a float32 or bfloat16 torch CUDA tensor.  See include/eco.h."""
+    import torch
+    c = cfg.c()
+    st = load_library().eco_dequantize(ctypes.byref(c), _addr(w), _addr(scale), rows, cols, _addr(out),
+                                       1 if out.dtype == torch.bfloat16 else 0, device, stream)
     if st != ECO_OK:
         _raise(st)
 

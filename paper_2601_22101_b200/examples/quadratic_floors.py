@@ -25,8 +25,15 @@ import torch
 from .. import eco
 
 
+_FP8_TENSOR = eco.Config(format=eco.ECO_FORMAT_FP8_E4M3, granularity=eco.ECO_SCALE_PER_TENSOR, scale_dtype=eco.ECO_SCALE_F32)
+
+
 def _dequant(codes: torch.Tensor, scale: torch.Tensor) -> torch.Tensor:
-    return codes.view(torch.float8_e4m3fn).to(torch.float32) * scale
+    """The weights the "forward pass" sees: value(code) * scale, expanded by the library."""
+    out = torch.empty(codes.numel(), dtype=torch.float32, device=codes.device)
+    eco.eco_dequantize(_FP8_TENSOR, codes, scale, 1, codes.numel(), out, device=codes.device.index or 0,
+                       stream=torch.cuda.current_stream(codes.device).cuda_stream)
+    return out
 
 
 def run(regime: str, lr: float, steps: int, n_rows: int = 256, cols: int = 1024, beta: float = 0.9,

@@ -469,3 +469,28 @@ def test_error_buffers_and_exact_injection(fmt, gran, rnd, injection):
                 assert (ebufs[i].cpu().numpy().view(np.int32) == ora.e[i].view(np.int32)).all(), f"step {step} tensor {i}: error buffer"
     finally:
         dev.destroy()
+
+
+@pytest.mark.parametrize("fmt,sdt", [(wl.FP8_E4M3, wl.SCALE_F32), (wl.INT4, wl.SCALE_BF16), (wl.FP8_E4M3, wl.SCALE_BF16)])
+@pytest.mark.parametrize("gran", [wl.PER_BLOCK, wl.PER_TENSOR, wl.PER_ROW])
+def test_dequantize_parity(fmt, sdt, gran):
+    """eco_dequantize (f32 exact, bf16 nearest-even) against the oracle's dequantizer on ragged shapes."""
+    rng = np.random.default_rng(3)
+    w = _mini(fmt, gran, sdt, wl.SGDM, wl.RTN, RAGGED + (RAGGED_FP8_ONLY if fmt == wl.FP8_E4M3 else []))
+    cfg_o, cfg_d = oracle_config(w), config_of(w)
+    for t in w.tensors:
+        x = (rng.standard_normal((t.rows, t.cols)) * 0.02).astype(np.float32)
+        ow, os_ = oracle.quantize(cfg_o, x)
+        ref = oracle.dequantize(cfg_o, ow, os_, t.rows, t.cols)
+        dw = torch.from_numpy(ow).cuda()
+        ds = torch.from_numpy(os_.view(np.int16) if os_.dtype == np.uint16 else os_).cuda()
+        if os_.dtype == np.uint16:
+            ds = ds.view(torch.bfloat16)
+        out32 = torch.zeros(t.numel, dtype=torch.float32, device="cuda")
+        out16 = torch.zeros(t.numel, dtype=torch.bfloat16, device="cuda")
+        eco.eco_dequantize(cfg_d, dw, ds, t.rows, t.cols, out32)
+        eco.eco_dequantize(cfg_d, dw, ds, t.rows, t.cols, out16)
+        torch.cuda.synchronize()
+        assert (out32.cpu().numpy().view(np.int32) == ref.reshape(-1).view(np.int32)).all(), (t.rows, t.cols)
+        expect16 = torch.from_numpy(ref.reshape(-1)).to(torch.bfloat16)
+        assert torch.equal(out16.cpu().view(torch.int16), expect16.view(torch.int16)), (t.rows, t.cols)
