@@ -192,6 +192,7 @@ StepParams derive_params(const eco_config& cfg, float lr_f, float beta1_f, float
     P.grad_scale = grad_scale_f;
     P.has_decay = weight_decay_f != 0.0f ? 1 : 0;
     P.has_grad_scale = grad_scale_f != 1.0f ? 1 : 0;
+    P.fast_ok = (eps_f >= 0.0f && eps_f <= 1073741824.0f) ? 1 : 0;
     P.alpha = static_cast<float>((1.0 / lr) * (1.0 - 1.0 / b1));
     if (cfg.optimizer == ECO_OPT_ADAM) {
         const double bc1 = 1.0 - std::pow(b1, t);

@@ -205,6 +205,13 @@ def c3_rowwise() -> Workload:
     return replace(w, name="c3_gemma3_1b_fp8_row_adam_sr", granularity=PER_ROW)
 
 
+def c5_tensorwise_adam() -> Workload:
+    """The DeepSeek-MoE-shaped expert set the way the paper fine-tuned it (Sec. 4.5): tensor-wise INT4, Adam."""
+    w = c5()
+    return replace(w, name="c5_deepseek_moe16b_int4_tensor_adam_sr", granularity=PER_TENSOR, scale_dtype=SCALE_F32,
+                   optimizer=ADAM, beta2=0.95, eps=1e-8)
+
+
 def c4_small() -> Workload:
     """One layer (64 experts) of the sparse-MoE set (profiling-sized: ~1.5 GB of state)."""
     w = c4(layers=1)
@@ -247,7 +254,14 @@ def replicate(w: Workload, copies: int) -> Workload:
     return replace(w, name=f"{w.name}_x{copies}", tensors=ts)
 
 
-BY_NAME = {"c1": c1, "c2": c2, "c3": c3, "c4": c4, "c5": c5, "c3r": c3_rowwise,
+def c4_dense() -> Workload:
+    """The sparse-MoE set with EVERY expert receiving a gradient (no all-zero gradients): the dense-gradient rate of
+    the FP8 1x128 Adam path at 2.1B parameters."""
+    w = c4()
+    return replace(w, name="c4_smoe_2mat_fp8_block128_adam_sr_all_routed", tensors=[replace(t, zero_grad=False) for t in w.tensors])
+
+
+BY_NAME = {"c1": c1, "c2": c2, "c3": c3, "c4": c4, "c5": c5, "c3r": c3_rowwise, "c5t": c5_tensorwise_adam, "c4g": lambda: c4(expert_mats=3), "c4d": c4_dense,
            "c3s": c3_small, "c4s": c4_small, "c5s": c5_small}
 
 
