@@ -143,7 +143,9 @@ __device__ __forceinline__ bool consume_unit(const StepParams& P, const int bf16
             uint32_t codes = 0;
             float s_old = 1.0f;
 #pragma unroll
-            for (int e = 0; e < 4; ++e) { g[k][e] = 0.f; m[k][e] = 0.f; v[k][e] = 0.f; }
+            // rows that are not present (short units) carry harmless values: their results are never stored, and
+            // ones keep the thread on the straight-line square root / division path (zeros would not)
+            for (int e = 0; e < 4; ++e) { g[k][e] = 0.f; m[k][e] = 1.f; v[k][e] = 1.f; }
             if (valid) {
                 if (FMT == FMT_FP8) codes = *reinterpret_cast<const uint32_t*>(st + SL::kCodes + row * 128 + lane * 4);
                 else codes = *reinterpret_cast<const uint16_t*>(st + SL::kCodes + row * 64 + lane * 2);
