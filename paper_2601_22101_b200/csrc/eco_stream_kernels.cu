@@ -120,25 +120,30 @@ __device__ __forceinline__ uint32_t units_of(const TensorDesc& T) {
 
 // One unit (up to 32 rows of 128 elements) by the 8 consumer warps: warp w owns rows 4w..4w+3, lane l
 // elements 4l..4l+3 of each.  FULL: all 32 rows are present (every unit but the last of a tensor).
-template <int FMT, int OPT, int RND, int MODE, bool FULL, bool ERR>
+template <int FMT, int OPT, int RND, int MODE, bool FULL, bool ERR, int NS = 4>
 __device__ __forceinline__ bool consume_unit(const StepParams& P, const int bf16_scale, const uint8_t* st,
                                              const StageHeader* h, const uint32_t empty_bar, const int warp,
                                              const int lane, uint32_t* scratch_amax, uint32_t& cur_slot,
                                              float& run_max, float* xchg, const uint32_t row_bars,
                                              const uint32_t row_parity, uint32_t* status) {
     using SL = StageLayout<FMT, OPT>;
-    const int r = warp * 4;
-    const int nrows = FULL ? kUnitRows : static_cast<int>(h->nrows);
-    const uint64_t i_first = (h->row0 + r) * 128 + lane * 4;      // element index of (row r, this lane)
+    // Row (of 128 elements) behind slot k of this warp.  Per-row mode deals the rows round-robin (warp, warp + 8, ...)
+    // so that a unit of fewer than 32 rows leaves every warp with 3 or 4 rows instead of some with none; NS is the
+    // number of slots this instantiation carries (with FULL: all of them present).
+    static_assert(NS == 4 || MODE == MODE_ROW, "only the per-row mode runs with fewer slots");
+    constexpr int kRowStep = MODE == MODE_ROW ? kConsumerWarps : 1;
+    const int r = MODE == MODE_ROW ? warp : warp * 4;
+    const int nrows = static_cast<int>(h->nrows);
+    const uint64_t i_first = (h->row0 + r) * 128 + lane * 4;      // element index of (slot 0, this lane)
     float* const vp = h->v;
 
-    Lane4<OPT> L[4];
-    float amax[4];
+    Lane4<OPT> L[NS];
+    float amax[NS];
     {
-        float th[4][4], g[4][4], m[4][4], v[4][4], vt[4][4];
+        float th[NS][4], g[NS][4], m[NS][4], v[NS][4], vt[NS][4];
 #pragma unroll
-        for (int k = 0; k < 4; ++k) {
-            const int row = r + k;
+        for (int k = 0; k < NS; ++k) {
+            const int row = r + k * kRowStep;
             const bool valid = FULL || row < nrows;
             uint32_t codes = 0;
             float s_old = 1.0f;
@@ -167,14 +172,14 @@ __device__ __forceinline__ bool consume_unit(const StepParams& P, const int bf16
 #pragma unroll
             for (int e = 0; e < 4; ++e) th[k][e] = __fmul_rn(val[e], s_old);
         }
-        optim_rows<OPT, 4>(P, th, g, m, v, L, vt);
+        optim_rows<OPT, NS>(P, th, g, m, v, L, vt);
 #pragma unroll
-        for (int k = 0; k < 4; ++k) {
-            const bool valid = FULL || r + k < nrows;
+        for (int k = 0; k < NS; ++k) {
+            const bool valid = FULL || r + k * kRowStep < nrows;
             amax[k] = 0.0f;
             if (valid) amax[k] = fmaxf(fmaxf(fabsf(L[k].tht[0]), fabsf(L[k].tht[1])), fmaxf(fabsf(L[k].tht[2]), fabsf(L[k].tht[3])));
             if (OPT == OPT_ADAM && MODE != MODE_TENSOR_AMAX && valid)
-                *reinterpret_cast<float4*>(vp + i_first + k * 128) = make_float4(vt[k][0], vt[k][1], vt[k][2], vt[k][3]);
+                *reinterpret_cast<float4*>(vp + i_first + k * (kRowStep * 128)) = make_float4(vt[k][0], vt[k][1], vt[k][2], vt[k][3]);
         }
     }
     // everything needed later is read before the stage is handed back
@@ -199,11 +204,12 @@ __device__ __forceinline__ bool consume_unit(const StepParams& P, const int bf16
             cur_slot = slot;
             run_max = 0.0f;
         }
-        run_max = fmaxf(fmaxf(run_max, fmaxf(amax[0], amax[1])), fmaxf(amax[2], amax[3]));
+#pragma unroll
+        for (int k = 0; k < NS; ++k) run_max = fmaxf(run_max, amax[k]);
         return true;
     }
 
-    float s_k[4], inv_k[4];
+    float s_k[NS], inv_k[NS];
     if (MODE == MODE_BLOCK) {
         // row maxima: one warp reduction per row; lane group g = lane / 8 then derives the scale of row g
         // and the four scales are broadcast from lanes 0, 8, 16, 24
@@ -231,9 +237,9 @@ __device__ __forceinline__ bool consume_unit(const StepParams& P, const int bf16
         float* xs = xchg + 32;
         float* xinv = xchg + 64;
 #pragma unroll
-        for (int k = 0; k < 4; ++k) {
+        for (int k = 0; k < NS; ++k) {
             const float z = warp_amax(amax[k]);
-            if (lane == 0) xmax[r + k] = z;
+            if (lane == 0) xmax[r + k * kRowStep] = z;
         }
         __syncwarp();
         if (lane == 0) mbar_arrive(row_bars);
@@ -254,20 +260,20 @@ __device__ __forceinline__ bool consume_unit(const StepParams& P, const int bf16
         if (lane == 0) mbar_arrive(row_bars + 8);
         if (!mbar_wait(row_bars + 8, row_parity, status, 5u)) return false;
 #pragma unroll
-        for (int k = 0; k < 4; ++k) {
-            const uint32_t j = (static_cast<uint32_t>(r + k) * div_magic) >> 16;
-            const bool valid = FULL || r + k < nrows;
+        for (int k = 0; k < NS; ++k) {
+            const uint32_t j = (static_cast<uint32_t>(r + k * kRowStep) * div_magic) >> 16;
+            const bool valid = FULL || r + k * kRowStep < nrows;
             s_k[k] = valid ? xs[j] : 1.0f;
             inv_k[k] = valid ? xinv[j] : 1.0f;
         }
     } else {
 #pragma unroll
-        for (int k = 0; k < 4; ++k) { s_k[k] = s_new; inv_k[k] = inv_new; }
+        for (int k = 0; k < NS; ++k) { s_k[k] = s_new; inv_k[k] = inv_new; }
     }
 #pragma unroll
-    for (int k = 0; k < 4; ++k) {
-        if (!FULL && r + k >= nrows) continue;
-        const uint64_t i0 = i_first + k * 128;
+    for (int k = 0; k < NS; ++k) {
+        if (!FULL && r + k * kRowStep >= nrows) continue;
+        const uint64_t i0 = i_first + k * (kRowStep * 128);
         uint32_t word[4] = {0u, 0u, 0u, 0u};
         if (RND == RND_SR) {
             const uint4 rw = philox4x32_10(static_cast<uint32_t>((i0 + index_base) >> 2), tensor_id, P.step_lo, P.step_hi, P);
@@ -440,12 +446,24 @@ eco_stream_kernel(const TensorDesc* __restrict__ descs, const uint32_t* __restri
         const uint32_t nrows = h->nrows;
         if (nrows == 0u) break;                   // end marker
         bool ok;
-        if (nrows == kUnitRows)
+        if constexpr (MODE == MODE_ROW) {
+            // rows are dealt round-robin: this warp has rows warp, warp + 8, ... below nrows
+            const int mine = static_cast<int>(nrows) > warp ? (static_cast<int>(nrows) - warp + kConsumerWarps - 1) / kConsumerWarps : 0;
+            if (mine == 4)
+                ok = consume_unit<FMT, OPT, RND, MODE, true, ERR, 4>(P, bf16_scale, st, h, empty, warp, lane, scratch_amax, cur_slot,
+                                                                     run_max, xchg, row_bars, it & 1u, status);
+            else if (mine == 3)
+                ok = consume_unit<FMT, OPT, RND, MODE, true, ERR, 3>(P, bf16_scale, st, h, empty, warp, lane, scratch_amax, cur_slot,
+                                                                     run_max, xchg, row_bars, it & 1u, status);
+            else
+                ok = consume_unit<FMT, OPT, RND, MODE, false, ERR, 4>(P, bf16_scale, st, h, empty, warp, lane, scratch_amax, cur_slot,
+                                                                      run_max, xchg, row_bars, it & 1u, status);
+        } else if (nrows == kUnitRows)   // (discarded statement of the if constexpr above for the per-row mode)
             ok = consume_unit<FMT, OPT, RND, MODE, true, ERR>(P, bf16_scale, st, h, empty, warp, lane, scratch_amax, cur_slot,
-                                                         run_max, xchg, row_bars, it & 1u, status);
+                                                              run_max, xchg, row_bars, it & 1u, status);
         else
             ok = consume_unit<FMT, OPT, RND, MODE, false, ERR>(P, bf16_scale, st, h, empty, warp, lane, scratch_amax, cur_slot,
-                                                          run_max, xchg, row_bars, it & 1u, status);
+                                                               run_max, xchg, row_bars, it & 1u, status);
         if (!ok) return;
     }
     if (MODE == MODE_TENSOR_AMAX && cur_slot != 0xFFFFFFFFu) {
