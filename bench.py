@@ -253,7 +253,7 @@ def main():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=5)
-    ap.add_argument("--workload", default="c4", choices=["c1", "c2", "c3", "c4", "c5", "c3r", "c5t", "c4g", "c4d", "c3s", "c4s", "c5s"])
+    ap.add_argument("--workload", default="c4", choices=["c1", "c2", "c3", "c4", "c5", "c3r", "c5t", "c4g", "c4d", "c3s", "c3rs", "c4s", "c5s"])
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--also", default="c3,c5", help="comma-separated workloads timed after the headline one and "
                     "reported under other_workloads (device-resident timing only)")

@@ -212,6 +212,12 @@ def c5_tensorwise_adam() -> Workload:
                    optimizer=ADAM, beta2=0.95, eps=1e-8)
 
 
+def c3_rowwise_small() -> Workload:
+    """c3_small with one scale per row (profiling-sized)."""
+    w = c3_small()
+    return replace(w, name="c3_gemma3_1b_fp8_row_adam_sr_small", granularity=PER_ROW)
+
+
 def c4_small() -> Workload:
     """One layer (64 experts) of the sparse-MoE set (profiling-sized: ~1.5 GB of state)."""
     w = c4(layers=1)
@@ -262,7 +268,7 @@ def c4_dense() -> Workload:
 
 
 BY_NAME = {"c1": c1, "c2": c2, "c3": c3, "c4": c4, "c5": c5, "c3r": c3_rowwise, "c5t": c5_tensorwise_adam, "c4g": lambda: c4(expert_mats=3), "c4d": c4_dense,
-           "c3s": c3_small, "c4s": c4_small, "c5s": c5_small}
+           "c3s": c3_small, "c3rs": c3_rowwise_small, "c4s": c4_small, "c5s": c5_small}
 
 
 def _rng(w: Workload, t: TensorSpec, step: int, kind: int) -> np.random.Generator:
