@@ -61,8 +61,13 @@ def load_library() -> ctypes.CDLL:
     global _lib
     if _lib is None:
         if not os.path.exists(_LIB_PATH):
-            raise ImportError(f"{_LIB_PATH} is missing: run `python -m paper_2601_22101_b200.build` "
-                              "(there is no CPU fallback)")
+            # not built yet: compile it now if nvcc is available; there is no other implementation to fall back to
+            try:
+                from . import build as _build
+                _build.build()
+            except Exception as exc:
+                raise ImportError(f"{_LIB_PATH} is missing and could not be built ({exc}): run "
+                                  "`python -m paper_2601_22101_b200.build` (there is no CPU fallback)") from exc
         L = ctypes.CDLL(_LIB_PATH)
         vp, u64, u32, i64, f32 = ctypes.c_void_p, ctypes.c_uint64, ctypes.c_uint32, ctypes.c_int64, ctypes.c_float
         L.eco_create.restype = ctypes.c_int
