@@ -19,7 +19,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 _SRC = os.path.join(_HERE, "eco_oracle.cpp")
 _LIB = os.path.join(_HERE, "libeco_oracle.so")
 
-FP8_E4M3, INT4, IDENTITY, ADDITIVE_NOISE = 0, 1, 2, 3
+FP8_E4M3, INT4, IDENTITY, ADDITIVE_NOISE, FP8_E5M2 = 0, 1, 2, 3, 4
 PER_TENSOR, PER_ROW, PER_BLOCK = 0, 1, 2
 SCALE_NATIVE, SCALE_BF16 = 0, 1
 SGDM, ADAM = 0, 1
@@ -67,7 +67,7 @@ class Config:
 
     def code_bytes(self, rows: int, cols: int) -> int:
         n = rows * cols
-        return n if self.format == FP8_E4M3 else (n + 1) // 2
+        return (n + 1) // 2 if self.format == INT4 else n
 
 
 _lib = None

@@ -36,7 +36,9 @@ namespace {
 // ---------------------------------------------------------------------------
 // Enumerations of the boundary (values shared with the C-ABI by number only).
 // ---------------------------------------------------------------------------
-enum Format { FMT_FP8_E4M3 = 0, FMT_INT4 = 1, FMT_IDENTITY = 2, FMT_ADDITIVE_NOISE = 3 };
+enum Format { FMT_FP8_E4M3 = 0, FMT_INT4 = 1, FMT_IDENTITY = 2, FMT_ADDITIVE_NOISE = 3, FMT_FP8_E5M2 = 4 };
+
+bool is_fp8(int format) { return format == FMT_FP8_E4M3 || format == FMT_FP8_E5M2; }
 enum Granularity { GRAN_TENSOR = 0, GRAN_ROW = 1, GRAN_BLOCK = 2 };
 enum ScaleDtype { SCALE_NATIVE = 0, SCALE_BF16 = 1 };  // native = R
 enum Optimizer { OPT_SGDM = 0, OPT_ADAM = 1 };
@@ -111,10 +113,13 @@ uint16_t f32_to_bf16_rne(float f) {
 // FP8-E4M3 is the OCP "FN" flavour: 1 sign, 4 exponent (bias 7), 3 mantissa
 // bits, no infinities, S.1111.111 is NaN, largest finite 448 = S.1111.110.
 // INT4 is the symmetric integer grid -7..7 (two's complement nibble, -8 unused).
+// FP8-E5M2 (the other OCP 8-bit float, offered as a further format on the same skeleton: Sec. 3.1 leaves the
+// format open): 1 sign, 5 exponent (bias 15), 2 mantissa bits, IEEE-style infinities and NaNs (never written),
+// largest finite 57344 = S.11110.11, subnormals M * 2^-16.
 // ---------------------------------------------------------------------------
 template <class R>
 R format_rho(int format) {
-    return format == FMT_FP8_E4M3 ? R(448) : R(7);
+    return format == FMT_FP8_E4M3 ? R(448) : (format == FMT_FP8_E5M2 ? R(57344) : R(7));
 }
 
 // Magnitude of a 7-bit E4M3 magnitude code (sign stripped).
@@ -126,8 +131,21 @@ R e4m3_magnitude(int mag_code) {
     return std::ldexp(R(1) + R(M) / R(8), E - 7);             // 2^(E-7) * (1 + M/8)
 }
 
+// Magnitude of a 7-bit E5M2 magnitude code (sign stripped).
+template <class R>
+R e5m2_magnitude(int mag_code) {
+    const int E = (mag_code >> 2) & 31, M = mag_code & 3;
+    if (E == 31) return M == 0 ? std::numeric_limits<R>::infinity() : std::numeric_limits<R>::quiet_NaN();
+    if (E == 0) return std::ldexp(R(M), -16);                 // subnormal: M * 2^-16
+    return std::ldexp(R(1) + R(M) / R(4), E - 15);            // 2^(E-15) * (1 + M/4)
+}
+
 template <class R>
 R code_value(int format, int code) {
+    if (format == FMT_FP8_E5M2) {
+        const R mag = e5m2_magnitude<R>(code & 0x7F);
+        return (code & 0x80) ? -mag : mag;
+    }
     if (format == FMT_FP8_E4M3) {
         const R mag = e4m3_magnitude<R>(code & 0x7F);
         return (code & 0x80) ? -mag : mag;
@@ -146,8 +164,11 @@ void lower_neighbour(int format, R a, int* lo_code, R* frac) {
         *frac = a - k;
         return;
     }
-    if (a < std::ldexp(R(1), -6)) {          // subnormal range, spacing 2^-9
-        const R q = std::ldexp(a, 9);
+    // binary floating-point grids: mb mantissa bits, smallest normal 2^emin, subnormal spacing 2^(emin - mb)
+    const int mb = format == FMT_FP8_E5M2 ? 2 : 3;
+    const int emin = format == FMT_FP8_E5M2 ? -14 : -6;
+    if (a < std::ldexp(R(1), emin)) {
+        const R q = std::ldexp(a, mb - emin);
         const R k = std::floor(q);
         *lo_code = static_cast<int>(k);
         *frac = q - k;
@@ -156,9 +177,9 @@ void lower_neighbour(int format, R a, int* lo_code, R* frac) {
     int ex;
     std::frexp(a, &ex);                       // a = f * 2^ex, f in [0.5, 1)
     const int e = ex - 1;                     // 2^e <= a < 2^(e+1)
-    const R q = std::ldexp(a, 3 - e);         // in [8, 16): spacing 2^(e-3)
+    const R q = std::ldexp(a, mb - e);        // in [2^mb, 2^(mb+1)): spacing 2^(e-mb)
     const R k = std::floor(q);
-    *lo_code = ((e + 7) << 3) | (static_cast<int>(k) - 8);
+    *lo_code = ((e - emin + 1) << mb) | (static_cast<int>(k) - (1 << mb));
     *frac = q - k;
 }
 
@@ -185,7 +206,7 @@ int round_to_code(int format, int rounding, R y, uint32_t random_word) {
         up = (frac > R(0.5)) || (frac == R(0.5) && (lo & 1));
     }
     const int mag = lo + (up ? 1 : 0);
-    if (format == FMT_FP8_E4M3) return (negative ? 0x80 : 0) | mag;
+    if (is_fp8(format)) return (negative ? 0x80 : 0) | mag;
     return (negative ? -mag : mag) & 0xF;
 }
 
@@ -194,13 +215,13 @@ int round_to_code(int format, int rounding, R y, uint32_t random_word) {
 // byte, element 2k in the low nibble) and scales (R, or bf16 when R = float).
 // ---------------------------------------------------------------------------
 int load_code(int format, const uint8_t* w, uint64_t i) {
-    if (format == FMT_FP8_E4M3) return w[i];
+    if (is_fp8(format)) return w[i];
     const uint8_t byte = w[i >> 1];
     return (i & 1) ? (byte >> 4) : (byte & 0xF);
 }
 
 void store_code(int format, uint8_t* w, uint64_t i, int code) {
-    if (format == FMT_FP8_E4M3) { w[i] = static_cast<uint8_t>(code); return; }
+    if (is_fp8(format)) { w[i] = static_cast<uint8_t>(code); return; }
     uint8_t& byte = w[i >> 1];
     if (i & 1) byte = static_cast<uint8_t>((byte & 0x0F) | ((code & 0xF) << 4));
     else       byte = static_cast<uint8_t>((byte & 0xF0) | (code & 0xF));
@@ -382,7 +403,7 @@ int step_tensor(const OracleConfig& cfg, const Hyper& hyper,
                 uint64_t rows, uint64_t cols, uint32_t tensor_id,
                 const R* noise, R* e_prev, R* dbg_theta_tilde, R* dbg_err) {
     const StepScalars<R> sc = derive_scalars<R>(hyper);
-    const bool coded = cfg.format == FMT_FP8_E4M3 || cfg.format == FMT_INT4;
+    const bool coded = is_fp8(cfg.format) || cfg.format == FMT_INT4;
     OracleConfig grid_cfg = cfg;
     if (!coded) grid_cfg.granularity = GRAN_TENSOR;
     const BlockGrid g = block_grid(grid_cfg, rows, cols);

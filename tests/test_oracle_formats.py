@@ -146,3 +146,65 @@ def test_bf16_rounding_matches_library():
     ref = torch.from_numpy(x).to(torch.bfloat16).view(torch.int16).numpy().astype(np.uint16)
     got = np.array([oracle.f32_to_bf16(v) for v in x], dtype=np.uint16)
     assert (got == ref).all()
+
+
+# --------------------------------------------------------------------------- FP8-E5M2 (a further format on the same skeleton)
+def _e5m2_closed_form(code: int) -> float:
+    s, E, M = code >> 7, (code >> 2) & 31, code & 3
+    if E == 31:
+        mag = math.inf if M == 0 else math.nan
+    else:
+        mag = M * 2.0 ** -16 if E == 0 else 2.0 ** (E - 15) * (1 + M / 4)
+    return -mag if s else mag
+
+
+def test_e5m2_decode_all_codes_closed_form_and_library():
+    from oracle import FP8_E5M2
+    lib_vals = torch.arange(256, dtype=torch.uint8).view(torch.float8_e5m2).to(torch.float64).numpy()
+    for c in range(256):
+        v, ref = oracle.code_value(FP8_E5M2, c), _e5m2_closed_form(c)
+        if math.isnan(ref):
+            assert math.isnan(v) and math.isnan(lib_vals[c])
+        else:
+            assert v == ref == lib_vals[c], c
+    assert oracle.code_value(FP8_E5M2, 0x7B) == 57344.0       # rho: largest finite magnitude
+    assert oracle.code_value(FP8_E5M2, 0x01) == 2.0 ** -16    # smallest subnormal
+    assert oracle.code_value(FP8_E5M2, 0x04) == 2.0 ** -14    # smallest normal
+
+
+def test_e5m2_round_trip_midpoints_saturation_and_library_cast():
+    from oracle import FP8_E5M2
+    mags = [oracle.code_value(FP8_E5M2, c) for c in range(0x7C)]          # finite magnitudes
+    assert all(b > a for a, b in zip(mags, mags[1:]))
+    for dtype in (np.float32, np.float64):
+        y = np.array(mags + [-m for m in mags], dtype=dtype)
+        codes = oracle.round_to_codes(FP8_E5M2, RTN, y)
+        assert list(codes[:0x7C]) == list(range(0x7C)) and list(codes[0x7C:]) == [0x80 | c for c in range(0x7C)]
+        for r in (0, 0xFFFFFFFF):
+            assert (oracle.round_to_codes(FP8_E5M2, SR, y, np.full(y.size, r, np.uint32)) == codes).all()
+    for c in range(0x7B):                                                    # midpoints go to the even code
+        mid = (mags[c] + mags[c + 1]) / 2
+        even = c if c % 2 == 0 else c + 1
+        got = oracle.round_to_codes(FP8_E5M2, RTN, np.array([mid, np.nextafter(np.float32(mid), np.float32(0)),
+                                                             np.nextafter(np.float32(mid), np.float32(1e9))], np.float32))
+        assert list(got) == [even, c, c + 1], c
+    big = np.array([57344.0, 60000.0, 1e9, np.inf, -1e9, np.nan], np.float32)   # saturate, never inf / NaN codes
+    assert list(oracle.round_to_codes(FP8_E5M2, RTN, big)) == [0x7B, 0x7B, 0x7B, 0x7B, 0xFB, 0x7B]
+    rng = np.random.default_rng(5)
+    y = np.concatenate([rng.standard_normal(20000) * s for s in (1e-6, 1e-3, 1.0, 1e3)]).astype(np.float32)
+    y = y[np.abs(y) < 57344]
+    lib = torch.from_numpy(y).to(torch.float8_e5m2).view(torch.uint8).numpy()
+    assert (oracle.round_to_codes(FP8_E5M2, RTN, y) == lib).all()
+
+
+def test_e5m2_sr_probability_by_enumeration():
+    from oracle import FP8_E5M2
+    lo, gap = 1.25, 0.25                                     # between codes 1.25 and 1.5 (binade [1, 2), spacing 1/4)
+    for frac in (0.0, 2.0 ** -21, 0.3, 0.5, 1 - 2.0 ** -21):
+        y = np.float32(lo + frac * gap)
+        f = (float(y) - lo) / gap
+        words = (np.arange(0, 1 << 24, 4099, dtype=np.uint64) << 8).astype(np.uint32)
+        codes = oracle.round_to_codes(FP8_E5M2, SR, np.full(words.size, y, np.float32), words)
+        up = codes != oracle.round_to_codes(FP8_E5M2, RTN, np.array([lo], np.float32))[0]
+        expect = (words >> 8).astype(np.float64) < f * 2 ** 24
+        assert (up == expect).all()
