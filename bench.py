@@ -50,7 +50,7 @@ def _dominant_kernel(w) -> str:
     """Name of the kernel that moves most of a step's bytes (full-size sets are made of whole 128-element rows,
     which the persistent TMA-fed kernel takes)."""
     from paper_2601_22101_b200 import workloads as wl
-    fmt = "fp8" if w.format == wl.FP8_E4M3 else "int4"
+    fmt = {wl.FP8_E4M3: "fp8", wl.INT4: "int4", wl.FP8_E5M2: "e5m2"}[w.format]
     opt = "adam" if w.optimizer == wl.ADAM else "sgdm"
     rnd = "sr" if w.rounding == wl.SR else "rtn"
     mode = {wl.PER_BLOCK: "block", wl.PER_TENSOR: "tensor_apply", wl.PER_ROW: "row"}[w.granularity]
@@ -64,7 +64,7 @@ def _two_pass_note(w, params, ms_per_step, peak):
     from paper_2601_22101_b200 import workloads as wl
     if w.granularity != wl.PER_TENSOR:
         return {}
-    code = 1.0 if w.format == wl.FP8_E4M3 else 0.5
+    code = 0.5 if w.format == wl.INT4 else 1.0
     moments = 4.0 * (2 if w.optimizer == wl.ADAM else 1)
     moved = 2 * (code + 2.0 + moments) + (code + moments)
     gbs = params * moved / (ms_per_step * 1e-3) / 1e9
@@ -214,7 +214,7 @@ def run_e2e(w, device: int, steps: int, max_host_gb: float):
     from paper_2601_22101_b200 import eco, workloads as wl
     from paper_2601_22101_b200.state import config_of
     adam = w.optimizer == wl.ADAM
-    per_param = (1.0 if w.format == wl.FP8_E4M3 else 0.5) + 2 + (8 if adam else 4)
+    per_param = (0.5 if w.format == wl.INT4 else 1.0) + 2 + (8 if adam else 4)
     picked, total = [], 0
     for t in w.tensors:
         if (total + t.numel) * per_param > max_host_gb * 2 ** 30 and picked:

@@ -40,8 +40,11 @@ typedef enum eco_status {
 /* Weight format (Sec. 3.1; rho = largest representable magnitude). */
 enum { ECO_FORMAT_FP8_E4M3 = 0, /* OCP E4M3 "FN": bias 7, rho = 448, S.1111.111 = NaN is never written;
                                    one byte per element */
-       ECO_FORMAT_INT4 = 1 };   /* integers -7..7, rho = 7, two's-complement nibbles, two per byte,
+       ECO_FORMAT_INT4 = 1,     /* integers -7..7, rho = 7, two's-complement nibbles, two per byte,
                                    element 2k in the low nibble; -8 is never written */
+       ECO_FORMAT_FP8_E5M2 = 4 };/* OCP E5M2: bias 15, rho = 57344, infinities and NaNs are never written; one byte per
+                                   element.  Not used by the paper; offered because Sec. 3.1 holds for any format
+                                   with a largest magnitude rho */
 /* Scale granularity (Sec. 3.1, "granularity").  Tensors are row-major [rows, cols]. */
 enum { ECO_SCALE_PER_TENSOR = 0, /* 1 scale                                              */
        ECO_SCALE_PER_ROW = 1,    /* rows scales                                          */

@@ -91,7 +91,7 @@ eco_status fail(eco_ctx* ctx, eco_status st, const char* fmt, ...) {
 
 eco_status check_config(const eco_config* cfg, bool need_optimizer) {
     if (!cfg) return fail(nullptr, ECO_ERR_INVALID_ARG, "cfg is NULL");
-    if (cfg->format != ECO_FORMAT_FP8_E4M3 && cfg->format != ECO_FORMAT_INT4)
+    if (cfg->format != ECO_FORMAT_FP8_E4M3 && cfg->format != ECO_FORMAT_INT4 && cfg->format != ECO_FORMAT_FP8_E5M2)
         return fail(nullptr, ECO_ERR_UNSUPPORTED, "unknown format %d", cfg->format);
     if (cfg->granularity < ECO_SCALE_PER_TENSOR || cfg->granularity > ECO_SCALE_PER_BLOCK)
         return fail(nullptr, ECO_ERR_UNSUPPORTED, "unknown granularity %d", cfg->granularity);
@@ -115,7 +115,7 @@ eco_status check_config(const eco_config* cfg, bool need_optimizer) {
 
 LaunchConfig launch_config(const eco_config& cfg) {
     LaunchConfig lc;
-    lc.format = cfg.format == ECO_FORMAT_FP8_E4M3 ? eco::FMT_FP8 : eco::FMT_INT4;
+    lc.format = cfg.format == ECO_FORMAT_FP8_E4M3 ? eco::FMT_FP8 : (cfg.format == ECO_FORMAT_FP8_E5M2 ? eco::FMT_E5M2 : eco::FMT_INT4);
     lc.optimizer = cfg.optimizer == ECO_OPT_ADAM ? eco::OPT_ADAM : eco::OPT_SGDM;
     lc.rounding = cfg.rounding == ECO_ROUND_STOCHASTIC ? eco::RND_SR : eco::RND_RTN;
     lc.bf16_scale = cfg.scale_dtype == ECO_SCALE_BF16 ? 1 : 0;
@@ -129,7 +129,7 @@ uint64_t n_scales(const eco_config& cfg, int64_t rows, int64_t cols) {
 }
 
 uint64_t code_bytes(const eco_config& cfg, uint64_t numel) {
-    return cfg.format == ECO_FORMAT_FP8_E4M3 ? numel : (numel + 1) / 2;
+    return cfg.format == ECO_FORMAT_INT4 ? (numel + 1) / 2 : numel;
 }
 
 uint64_t scale_bytes(const eco_config& cfg, int64_t rows, int64_t cols) {
@@ -374,7 +374,7 @@ eco_status eco_create(eco_ctx** out, const eco_config* cfg, const eco_tensor* te
         // that pass 2 finds what pass 1 read still cached.
         int64_t budget = g_options.l2_group_bytes;
         if (budget < 0) budget = static_cast<int64_t>(prop.l2CacheSize) / 2;
-        const double in_bytes_per_elem = (cfg->format == ECO_FORMAT_FP8_E4M3 ? 1.0 : 0.5) + 2.0 + (adam ? 8.0 : 4.0);
+        const double in_bytes_per_elem = (cfg->format == ECO_FORMAT_INT4 ? 0.5 : 1.0) + 2.0 + (adam ? 8.0 : 4.0);
         std::vector<size_t> group;
         double group_bytes = 0;
         // tensors made of whole 128-element rows go to the streaming kernels, the rest to the direct-load ones

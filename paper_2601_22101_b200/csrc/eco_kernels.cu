@@ -342,6 +342,7 @@ eco_quantize_kernel(const float* __restrict__ x, uint8_t* __restrict__ w, void* 
 // ---------------------------------------------------------------------------
 #define ECO_DISPATCH_FMT(fmt, ...)                                   \
     if ((fmt) == FMT_FP8) { constexpr int F = FMT_FP8; __VA_ARGS__ } \
+    else if ((fmt) == FMT_E5M2) { constexpr int F = FMT_E5M2; __VA_ARGS__ } \
     else { constexpr int F = FMT_INT4; __VA_ARGS__ }
 #define ECO_DISPATCH_OPT(opt, ...)                                    \
     if ((opt) == OPT_SGDM) { constexpr int O = OPT_SGDM; __VA_ARGS__ } \

@@ -52,7 +52,7 @@ static_assert(sizeof(StageHeader) <= 128, "header must fit its slot");
 
 template <int FMT, int OPT>
 struct StageLayout {
-    static constexpr int kCodeRow = FMT == FMT_FP8 ? 128 : 64;   // bytes of codes per row
+    static constexpr int kCodeRow = FMT == FMT_INT4 ? 64 : 128;  // bytes of codes per row
     static constexpr int kHeader = 0;
     static constexpr int kScales = 128;                          // kUnitRows floats
     static constexpr int kCodes = kScales + kUnitRows * 4;
@@ -152,7 +152,7 @@ __device__ __forceinline__ bool consume_unit(const StepParams& P, const int bf16
             // ones keep the thread on the straight-line square root / division path (zeros would not)
             for (int e = 0; e < 4; ++e) { g[k][e] = 0.f; m[k][e] = 1.f; v[k][e] = 1.f; }
             if (valid) {
-                if (FMT == FMT_FP8) codes = *reinterpret_cast<const uint32_t*>(st + SL::kCodes + row * 128 + lane * 4);
+                if (FMT != FMT_INT4) codes = *reinterpret_cast<const uint32_t*>(st + SL::kCodes + row * 128 + lane * 4);
                 else codes = *reinterpret_cast<const uint16_t*>(st + SL::kCodes + row * 64 + lane * 2);
                 const uint2 gr = *reinterpret_cast<const uint2*>(st + SL::kGrad + row * 256 + lane * 8);
                 g[k][0] = __uint_as_float(gr.x << 16); g[k][1] = __uint_as_float(gr.x & 0xFFFF0000u);
@@ -285,7 +285,7 @@ __device__ __forceinline__ bool consume_unit(const StepParams& P, const int bf16
             e_prev[0] = er.x; e_prev[1] = er.y; e_prev[2] = er.z; e_prev[3] = er.w;
         }
         const uint32_t codes = back4<FMT, OPT, RND, ERR>(P, word, s_k[k], inv_k[k], L[k], mh, e_prev, e_out);
-        if (FMT == FMT_FP8) *reinterpret_cast<uint32_t*>(wp + i0) = codes;
+        if (FMT != FMT_INT4) *reinterpret_cast<uint32_t*>(wp + i0) = codes;
         else *reinterpret_cast<uint16_t*>(wp + (i0 >> 1)) = static_cast<uint16_t>(codes);
         *reinterpret_cast<float4*>(mp + i0) = make_float4(mh[0], mh[1], mh[2], mh[3]);
         if (ERR) *reinterpret_cast<float4*>(ep + i0) = make_float4(e_out[0], e_out[1], e_out[2], e_out[3]);
@@ -494,6 +494,7 @@ static cudaError_t launch_one(const TensorDesc* descs, const uint32_t* unit_tens
 
 #define ECO_S_FMT(fmt, ...)                                            \
     if ((fmt) == FMT_FP8) { constexpr int F = FMT_FP8; __VA_ARGS__ }   \
+    else if ((fmt) == FMT_E5M2) { constexpr int F = FMT_E5M2; __VA_ARGS__ } \
     else { constexpr int F = FMT_INT4; __VA_ARGS__ }
 #define ECO_S_OPT(opt, ...)                                              \
     if ((opt) == OPT_SGDM) { constexpr int O = OPT_SGDM; __VA_ARGS__ }   \

@@ -17,7 +17,7 @@ _LIB_PATH = os.path.join(_HERE, "libeco_b200.so")
 # enum values of include/eco.h
 ECO_OK = 0
 ECO_ERR_INVALID_ARG, ECO_ERR_UNSUPPORTED, ECO_ERR_ALIGNMENT, ECO_ERR_CUDA, ECO_ERR_NOMEM, ECO_ERR_TIMEOUT = 1, 2, 3, 4, 5, 6
-ECO_FORMAT_FP8_E4M3, ECO_FORMAT_INT4 = 0, 1
+ECO_FORMAT_FP8_E4M3, ECO_FORMAT_INT4, ECO_FORMAT_FP8_E5M2 = 0, 1, 4
 ECO_SCALE_PER_TENSOR, ECO_SCALE_PER_ROW, ECO_SCALE_PER_BLOCK = 0, 1, 2
 ECO_SCALE_F32, ECO_SCALE_BF16 = 0, 1
 ECO_OPT_SGDM, ECO_OPT_ADAM = 0, 1

@@ -20,7 +20,7 @@ from typing import List, Optional
 import numpy as np
 
 # Enumerations of the C-ABI (include/eco.h), by value.
-FP8_E4M3, INT4 = 0, 1
+FP8_E4M3, INT4, FP8_E5M2 = 0, 1, 4
 PER_TENSOR, PER_ROW, PER_BLOCK = 0, 1, 2
 SCALE_F32, SCALE_BF16 = 0, 1
 SGDM, ADAM = 0, 1
@@ -74,17 +74,17 @@ class Workload:
         return t.rows * ((t.cols + self.block - 1) // self.block)
 
     def code_bytes(self, t: TensorSpec) -> int:
-        return t.numel if self.format == FP8_E4M3 else (t.numel + 1) // 2
+        return (t.numel + 1) // 2 if self.format == INT4 else t.numel
 
     def state_bytes_per_param(self) -> float:
         """Bytes of persistent state per parameter (codes + moments), scales excluded."""
-        w = 1.0 if self.format == FP8_E4M3 else 0.5
+        w = 0.5 if self.format == INT4 else 1.0
         return w + 4.0 + (4.0 if self.optimizer == ADAM else 0.0)
 
     def algorithmic_bytes_per_param(self) -> float:
         """Bytes one step must move per parameter: read codes, grad, moments and
         old scale; write codes, moments and new scale."""
-        w = 1.0 if self.format == FP8_E4M3 else 0.5
+        w = 0.5 if self.format == INT4 else 1.0
         moments = 4.0 * (2 if self.optimizer == ADAM else 1)
         n_scale = sum(self.n_scales(t) for t in self.tensors)
         sb = (4.0 if self.scale_dtype == SCALE_F32 else 2.0) * n_scale / max(self.numel, 1)

@@ -494,3 +494,29 @@ def test_dequantize_parity(fmt, sdt, gran):
         assert (out32.cpu().numpy().view(np.int32) == ref.reshape(-1).view(np.int32)).all(), (t.rows, t.cols)
         expect16 = torch.from_numpy(ref.reshape(-1)).to(torch.bfloat16)
         assert torch.equal(out16.cpu().view(torch.int16), expect16.view(torch.int16)), (t.rows, t.cols)
+
+
+@pytest.mark.parametrize("gran", [wl.PER_BLOCK, wl.PER_TENSOR, wl.PER_ROW])
+@pytest.mark.parametrize("opt", [wl.SGDM, wl.ADAM])
+@pytest.mark.parametrize("rnd", [wl.RTN, wl.SR])
+def test_e5m2_step_and_quantize_parity(rnd, opt, gran):
+    """The second 8-bit floating-point format (E5M2, rho = 57344) through the same kernels: chained steps on ragged
+    shapes, and eco_quantize on values that reach its subnormal range (below 2^-14 of the grid)."""
+    shapes = RAGGED + RAGGED_FP8_ONLY
+    run_chained(_mini(wl.FP8_E5M2, gran, wl.SCALE_F32, opt, rnd, shapes), steps=5)
+    rng = np.random.default_rng(8)
+    w = _mini(wl.FP8_E5M2, gran, wl.SCALE_F32, opt, rnd, [(7, 384), (3, 200)])
+    for t in w.tensors:
+        x = (rng.standard_normal((t.rows, t.cols)) * 0.02).astype(np.float32)
+        x.flat[:: 13] *= 1e-9          # 57344 * 1e-9 / amax-scale: deep in the subnormal range of the grid
+        x.flat[:: 31] = 0.0
+        ow, os_ = oracle.quantize(oracle_config(w), x, seed=7, step=2, tensor_id=t.tensor_id)
+        dw = torch.zeros(w.code_bytes(t), dtype=torch.uint8, device="cuda")
+        ds = torch.zeros(w.n_scales(t), dtype=torch.float32, device="cuda")
+        eco.eco_quantize(config_of(w), torch.from_numpy(x).cuda(), t.rows, t.cols, dw, ds, seed=7, step=2, tensor_id=t.tensor_id)
+        out = torch.zeros(t.numel, dtype=torch.float32, device="cuda")
+        eco.eco_dequantize(config_of(w), dw, ds, t.rows, t.cols, out)
+        torch.cuda.synchronize()
+        assert (_np(dw) == ow).all() and (_np(ds).view(np.int32) == os_.view(np.int32)).all()
+        ref = oracle.dequantize(oracle_config(w), ow, os_, t.rows, t.cols)
+        assert (_np(out).view(np.int32) == ref.reshape(-1).view(np.int32)).all()
