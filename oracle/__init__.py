@@ -21,7 +21,7 @@ _LIB = os.path.join(_HERE, "libeco_oracle.so")
 
 FP8_E4M3, INT4, IDENTITY, ADDITIVE_NOISE, FP8_E5M2 = 0, 1, 2, 3, 4
 PER_TENSOR, PER_ROW, PER_BLOCK = 0, 1, 2
-SCALE_NATIVE, SCALE_BF16 = 0, 1
+SCALE_NATIVE, SCALE_BF16, SCALE_E8M0 = 0, 1, 2
 SGDM, ADAM = 0, 1
 RTN, SR = 0, 1
 INJECT_NONE, INJECT_ECO, INJECT_IDEAL = 0, 1, 2
@@ -140,7 +140,7 @@ def round_to_codes(fmt: int, rounding: int, y: np.ndarray, r: np.ndarray | None 
 
 
 def scale_numpy_dtype(cfg: Config, real=np.float32):
-    return np.uint16 if cfg.scale_dtype == SCALE_BF16 else real
+    return {SCALE_BF16: np.uint16, SCALE_E8M0: np.uint8}.get(cfg.scale_dtype, real)
 
 
 def quantize(cfg: Config, x: np.ndarray, seed: int = 0, step: int = 0, tensor_id: int = 0):

@@ -22,7 +22,8 @@
 // by Monte Carlo; Philox against a library generator; identity quantizer ->
 // plain SGDM / Adam; Lemma 3.5 telescoping; the Adam one-step identity;
 // Appendix A exact equivalence with master weights; Appendix C stationary
-// second moments.  The order of the binary32 operations is this build's
+// second moments; power-of-two block scales against exact rational search,
+// a library decode of the exponent byte and power-of-two invariance.  The order of the binary32 operations is this build's
 // choice (the paper fixes none): parity unpinned for that order alone.
 
 #include <cmath>
@@ -40,7 +41,7 @@ enum Format { FMT_FP8_E4M3 = 0, FMT_INT4 = 1, FMT_IDENTITY = 2, FMT_ADDITIVE_NOI
 
 bool is_fp8(int format) { return format == FMT_FP8_E4M3 || format == FMT_FP8_E5M2; }
 enum Granularity { GRAN_TENSOR = 0, GRAN_ROW = 1, GRAN_BLOCK = 2 };
-enum ScaleDtype { SCALE_NATIVE = 0, SCALE_BF16 = 1 };  // native = R
+enum ScaleDtype { SCALE_NATIVE = 0, SCALE_BF16 = 1, SCALE_E8M0 = 2 };  // native = R; E8M0 = one byte, s = 2^(byte - 127)
 enum Optimizer { OPT_SGDM = 0, OPT_ADAM = 1 };
 enum Rounding { ROUND_RTN = 0, ROUND_SR = 1 };
 enum Injection { INJECT_NONE = 0, INJECT_ECO = 1, INJECT_IDEAL = 2 };
@@ -230,7 +231,23 @@ void store_code(int format, uint8_t* w, uint64_t i, int code) {
 template <class R>
 R load_scale(int scale_dtype, const void* scale, uint64_t k) {
     if (scale_dtype == SCALE_BF16) return R(bf16_to_f32(static_cast<const uint16_t*>(scale)[k]));
+    if (scale_dtype == SCALE_E8M0) return std::ldexp(R(1), static_cast<int>(static_cast<const uint8_t*>(scale)[k]) - 127);
     return static_cast<const R*>(scale)[k];
+}
+
+// Power-of-two scale (the shared-exponent scales of microscaling formats, which Sec. 3.1 cites among the group-wise
+// schemes): the smallest power of two s with s * rho >= amax, so that, like s = max|x| / rho, it prevents overflow;
+// exponent kept within what one byte with bias 127 holds (-127 .. 127; 0xFF is never written).
+template <class R>
+int pow2_scale_exponent(R amax, R rho) {
+    int e;
+    std::frexp(static_cast<long double>(amax / rho), &e);      // a first guess; the loops below decide exactly
+    if (e > 127) e = 127;
+    if (e < -127) e = -127;
+    const long double a = static_cast<long double>(amax), r = static_cast<long double>(rho);
+    while (e < 127 && std::ldexp(r, e) < a) ++e;
+    while (e > -127 && std::ldexp(r, e - 1) >= a) --e;
+    return e;
 }
 
 // Scale of a block with maximum magnitude amax (Sec. 3.1: s = max|x| / rho).
@@ -246,7 +263,13 @@ void make_scale(int format, int scale_dtype, R amax, void* scale, uint64_t k, R*
         s = R(1);
         inv = R(1);
         if (scale_dtype == SCALE_BF16) static_cast<uint16_t*>(scale)[k] = f32_to_bf16_rne(1.0f);
+        else if (scale_dtype == SCALE_E8M0) static_cast<uint8_t*>(scale)[k] = 127;
         else static_cast<R*>(scale)[k] = s;
+    } else if (scale_dtype == SCALE_E8M0) {
+        const int e = pow2_scale_exponent<R>(amax, rho);
+        static_cast<uint8_t*>(scale)[k] = static_cast<uint8_t>(e + 127);
+        s = std::ldexp(R(1), e);
+        inv = std::ldexp(R(1), -e);
     } else if (scale_dtype == SCALE_BF16) {
         const uint16_t h = f32_to_bf16_rne(static_cast<float>(amax / rho));
         static_cast<uint16_t*>(scale)[k] = h;

@@ -11,7 +11,7 @@ import torch
 
 import oracle
 from oracle import (ADAM, ADDITIVE_NOISE, FP8_E4M3, GRAD_BF16, GRAD_NATIVE, IDENTITY, INJECT_ECO, INJECT_IDEAL,
-                    INJECT_NONE, INT4, PER_BLOCK, PER_ROW, PER_TENSOR, RTN, SCALE_BF16, SCALE_NATIVE, SGDM, SR)
+                    INJECT_NONE, INT4, PER_BLOCK, PER_ROW, PER_TENSOR, RTN, SCALE_BF16, SCALE_E8M0, SCALE_NATIVE, SGDM, SR)
 
 GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
 
@@ -71,15 +71,16 @@ def test_sgdm_closed_form_one_step():
 # --------------------------------------------------------------------------- Lemma 3.5
 @pytest.mark.parametrize("fmt,gran,sdt,rnd", [
     (FP8_E4M3, PER_BLOCK, SCALE_NATIVE, SR), (FP8_E4M3, PER_TENSOR, SCALE_NATIVE, RTN),
-    (FP8_E4M3, PER_ROW, SCALE_NATIVE, SR), (INT4, PER_BLOCK, SCALE_BF16, SR), (INT4, PER_TENSOR, SCALE_NATIVE, RTN)])
+    (FP8_E4M3, PER_ROW, SCALE_NATIVE, SR), (INT4, PER_BLOCK, SCALE_BF16, SR), (INT4, PER_TENSOR, SCALE_NATIVE, RTN),
+    (FP8_E4M3, PER_BLOCK, SCALE_E8M0, SR), (INT4, PER_BLOCK, SCALE_E8M0, RTN)])
 def test_lemma_3_5_virtual_sequence_telescopes(fmt, gran, sdt, rnd):
     """theta_t := theta^_t - (eta beta/(1-beta)) m^_t obeys theta_{t+1} = theta_t - eta g_t for ANY
     quantizer, so over T steps it moves by -eta sum g.  Pins the error definition, the sign and the
     size of alpha (Eq. alpha) and that the new scale is the one the codes are read with."""
     rng = np.random.default_rng(11)
     rows, cols, lr, beta = 6, 200, 2e-3, 0.9
-    cfg = oracle.Config(format=fmt, granularity=gran, block=128, scale_dtype=sdt, optimizer=SGDM, rounding=rnd,
-                        grad_dtype=GRAD_NATIVE)
+    cfg = oracle.Config(format=fmt, granularity=gran, block=32 if sdt == SCALE_E8M0 else 128, scale_dtype=sdt,
+                        optimizer=SGDM, rounding=rnd, grad_dtype=GRAD_NATIVE)
     theta0 = rng.standard_normal((rows, cols)) * 0.02
     w, s = oracle.quantize(cfg, theta0)
     m = rng.standard_normal(rows * cols) * 1e-3
