@@ -222,7 +222,7 @@ def run_e2e(w, device: int, steps: int, max_host_gb: float):
         picked.append(t)
         total += t.numel
     ws = replace(w, tensors=picked)
-    sdt = torch.float32 if w.scale_dtype == wl.SCALE_F32 else torch.bfloat16
+    sdt = {wl.SCALE_F32: torch.float32, wl.SCALE_BF16: torch.bfloat16, wl.SCALE_E8M0: torch.uint8}[w.scale_dtype]
     tensors = []
     for t in ws.tensors:
         cw = torch.zeros(ws.code_bytes(t), dtype=torch.uint8).pin_memory()

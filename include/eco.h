@@ -51,7 +51,12 @@ enum { ECO_SCALE_PER_TENSOR = 0, /* 1 scale                                     
        ECO_SCALE_PER_BLOCK = 2 };/* rows * ceil(cols / block) scales, blocks of `block`
                                     consecutive elements of one row; the last block of a
                                     row may be short                                     */
-enum { ECO_SCALE_F32 = 0, ECO_SCALE_BF16 = 1 };
+/* Stored type of a scale.  F32: s = max|x| / rho.  BF16: that quotient rounded to bf16 (nearest even); the rounded
+ * value defines the grid.  E8M0: one byte b, s = 2^(b - 127), the smallest power of two with s * rho >= max|x|
+ * (so nothing overflows, as with s = max|x| / rho); b = 255 is never written, an all-zero block stores b = 127.
+ * The paper names power-of-two shared scales only by citation (Sec. 3.1, group-wise schemes); with block = 32 this is
+ * the layout of the microscaling formats. */
+enum { ECO_SCALE_F32 = 0, ECO_SCALE_BF16 = 1, ECO_SCALE_E8M0 = 2 };
 enum { ECO_OPT_SGDM = 0,  /* dampened momentum SGD: m~ = beta m + (1-beta) g, theta~ = theta^ - eta m~ (Eq. 2-3) */
        ECO_OPT_ADAM = 1 };/* Adam in the form of Sec. 3.2, "Adam"                                                */
 enum { ECO_ROUND_NEAREST = 0,    /* ties to the even code                                                        */
@@ -67,8 +72,8 @@ enum { ECO_INJECT_NONE = 0, /* naive master-weight removal (Sec. 3.4): the error
 typedef struct eco_config {
     int32_t format;      /* ECO_FORMAT_*                                  */
     int32_t granularity; /* ECO_SCALE_PER_*                               */
-    int32_t block;       /* block length for ECO_SCALE_PER_BLOCK: 128     */
-    int32_t scale_dtype; /* ECO_SCALE_F32 or ECO_SCALE_BF16               */
+    int32_t block;       /* block length for ECO_SCALE_PER_BLOCK: 128 or 32 */
+    int32_t scale_dtype; /* ECO_SCALE_F32, ECO_SCALE_BF16 or ECO_SCALE_E8M0 */
     int32_t optimizer;   /* ECO_OPT_*                                     */
     int32_t rounding;    /* ECO_ROUND_*                                   */
     int32_t injection;   /* ECO_INJECT_*; ECO_INJECT_ECO is the method    */

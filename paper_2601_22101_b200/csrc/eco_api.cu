@@ -95,9 +95,9 @@ eco_status check_config(const eco_config* cfg, bool need_optimizer) {
         return fail(nullptr, ECO_ERR_UNSUPPORTED, "unknown format %d", cfg->format);
     if (cfg->granularity < ECO_SCALE_PER_TENSOR || cfg->granularity > ECO_SCALE_PER_BLOCK)
         return fail(nullptr, ECO_ERR_UNSUPPORTED, "unknown granularity %d", cfg->granularity);
-    if (cfg->granularity == ECO_SCALE_PER_BLOCK && cfg->block != 128)
-        return fail(nullptr, ECO_ERR_UNSUPPORTED, "block %d: only 128 is built", cfg->block);
-    if (cfg->scale_dtype != ECO_SCALE_F32 && cfg->scale_dtype != ECO_SCALE_BF16)
+    if (cfg->granularity == ECO_SCALE_PER_BLOCK && cfg->block != 128 && cfg->block != 32)
+        return fail(nullptr, ECO_ERR_UNSUPPORTED, "block %d: 128 and 32 are built", cfg->block);
+    if (cfg->scale_dtype != ECO_SCALE_F32 && cfg->scale_dtype != ECO_SCALE_BF16 && cfg->scale_dtype != ECO_SCALE_E8M0)
         return fail(nullptr, ECO_ERR_UNSUPPORTED, "unknown scale_dtype %d", cfg->scale_dtype);
     if (cfg->rounding != ECO_ROUND_NEAREST && cfg->rounding != ECO_ROUND_STOCHASTIC)
         return fail(nullptr, ECO_ERR_UNSUPPORTED, "unknown rounding %d", cfg->rounding);
@@ -118,7 +118,9 @@ LaunchConfig launch_config(const eco_config& cfg) {
     lc.format = cfg.format == ECO_FORMAT_FP8_E4M3 ? eco::FMT_FP8 : (cfg.format == ECO_FORMAT_FP8_E5M2 ? eco::FMT_E5M2 : eco::FMT_INT4);
     lc.optimizer = cfg.optimizer == ECO_OPT_ADAM ? eco::OPT_ADAM : eco::OPT_SGDM;
     lc.rounding = cfg.rounding == ECO_ROUND_STOCHASTIC ? eco::RND_SR : eco::RND_RTN;
-    lc.bf16_scale = cfg.scale_dtype == ECO_SCALE_BF16 ? 1 : 0;
+    lc.scale_kind = cfg.scale_dtype == ECO_SCALE_BF16 ? eco::SCALE_KIND_BF16
+                    : (cfg.scale_dtype == ECO_SCALE_E8M0 ? eco::SCALE_KIND_E8M0 : eco::SCALE_KIND_F32);
+    lc.sub = (cfg.granularity == ECO_SCALE_PER_BLOCK && cfg.block == 32) ? 4 : 1;
     return lc;
 }
 
@@ -133,7 +135,7 @@ uint64_t code_bytes(const eco_config& cfg, uint64_t numel) {
 }
 
 uint64_t scale_bytes(const eco_config& cfg, int64_t rows, int64_t cols) {
-    return n_scales(cfg, rows, cols) * (cfg.scale_dtype == ECO_SCALE_BF16 ? 2 : 4);
+    return n_scales(cfg, rows, cols) * (cfg.scale_dtype == ECO_SCALE_BF16 ? 2 : (cfg.scale_dtype == ECO_SCALE_E8M0 ? 1 : 4));
 }
 
 eco_status check_shape(const eco_config& cfg, int64_t rows, int64_t cols, size_t i) {
@@ -313,6 +315,7 @@ eco_status eco_create(eco_ctx** out, const eco_config* cfg, const eco_tensor* te
         d.numel = static_cast<uint64_t>(t.rows) * static_cast<uint64_t>(t.cols);
         d.cols = static_cast<uint32_t>(t.cols);
         d.blocks_per_row = static_cast<uint32_t>((t.cols + 127) / 128);
+        d.scales_per_row = cfg->granularity == ECO_SCALE_PER_BLOCK ? static_cast<uint32_t>((t.cols + cfg->block - 1) / cfg->block) : 1u;
         d.tensor_id = t.tensor_id;
         d.slot = static_cast<uint32_t>(i);
         d.index_base = static_cast<uint64_t>(t.row_offset) * static_cast<uint64_t>(t.cols);
@@ -514,7 +517,7 @@ eco_status enqueue_step(eco_ctx* ctx, const StepParams& P, void* cuda_stream, in
         const uint32_t* units = ctx->d_unit_tensor + L.unit_offset;
         switch (L.kind) {
             case KIND_BLOCK_FAST:
-                ECO_CUDA(ctx, eco::launch_stream(ctx->lc, eco::STREAM_BLOCK, descs, units, L.n_units, P, nullptr, nullptr,
+                ECO_CUDA(ctx, eco::launch_stream(ctx->lc, ctx->lc.sub == 4 ? eco::STREAM_BLOCK32 : eco::STREAM_BLOCK, descs, units, L.n_units, P, nullptr, nullptr,
                                                  nullptr, false, ctx->d_tickets, ctx->d_status, ctx->grid_cap, stream, ctx->has_error_buffers));
                 break;
             case KIND_BLOCK_GENERIC:
@@ -639,7 +642,7 @@ eco_status eco_quantize(const eco_config* cfg, const float* x, int64_t rows, int
     } else {
         const uint64_t n_blocks = static_cast<uint64_t>(rows) * static_cast<uint64_t>((cols + 127) / 128);
         const uint32_t grid = static_cast<uint32_t>(std::min<uint64_t>(cap, (n_blocks + 7) / 8));
-        ECO_CUDA(nullptr, eco::launch_quantize(lc, x, static_cast<uint8_t*>(w), scale, rows, static_cast<uint32_t>(cols), 3, P, tensor_id, nullptr, grid, stream));
+        ECO_CUDA(nullptr, eco::launch_quantize(lc, x, static_cast<uint8_t*>(w), scale, rows, static_cast<uint32_t>(cols), lc.sub == 4 ? 4 : 3, P, tensor_id, nullptr, grid, stream));
     }
     return ECO_OK;
 }

@@ -70,16 +70,37 @@ __device__ __forceinline__ void row_extent(const TensorDesc& T, uint64_t blk, in
     vec = (start & 3) == 0;
 }
 
+// Maximum over each group of 8 lanes (one 32-element scale block); every lane of the group gets it.
+__device__ __forceinline__ float group8_max(float z) {
+    z = fmaxf(z, __shfl_xor_sync(0xFFFFFFFFu, z, 4));
+    z = fmaxf(z, __shfl_xor_sync(0xFFFFFFFFu, z, 2));
+    z = fmaxf(z, __shfl_xor_sync(0xFFFFFFFFu, z, 1));
+    return z;
+}
+
+// Index of the scale of 32-element block g (0..3) of 128-element chunk `blk`; the chunk's blocks that lie
+// inside the row are those with 128 j + 32 g < cols.
+template <bool GENERIC>
+__device__ __forceinline__ bool scale32_index(const TensorDesc& T, uint64_t blk, int g, uint64_t& k) {
+    if (blk >= T.n_blocks) return false;
+    if (!GENERIC) { k = blk * 4 + g; return true; }
+    const uint64_t row = blk / T.blocks_per_row;
+    const uint32_t j = static_cast<uint32_t>(blk - row * T.blocks_per_row);
+    k = row * T.scales_per_row + j * 4u + g;
+    return j * 128u + 32u * g < T.cols;
+}
+
 // ---------------------------------------------------------------------------
-// 1x128 block scales: the whole step in one pass.
-// GENERIC = false: cols is a multiple of 128, so scale block k is elements
-// 128k..128k+127 of the flat tensor.  GENERIC = true: any cols; the last block
+// Block scales along the row: the whole step in one pass.  A warp handles chunks of 128 consecutive elements
+// of a row; SUB = 1: the chunk is one scale block (1x128), SUB = 4: four blocks of 32 (8 lanes each).
+// GENERIC = false: cols is a multiple of 128, so chunk k is elements
+// 128k..128k+127 of the flat tensor.  GENERIC = true: any cols; the last chunk
 // of a row may be short and rows need not start on a 4-element boundary.
 // ---------------------------------------------------------------------------
-template <int FMT, int OPT, int RND, bool GENERIC>
+template <int FMT, int OPT, int RND, bool GENERIC, int SUB>
 __global__ void __launch_bounds__(kThreads)
 eco_block128_kernel(const TensorDesc* __restrict__ descs, const uint32_t* __restrict__ unit_tensor,
-                    const StepParams P, const int bf16_scale) {
+                    const StepParams P, const int scale_kind) {
     const uint32_t unit = blockIdx.x;
     const TensorDesc T = descs[unit_tensor[unit]];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -91,23 +112,43 @@ eco_block128_kernel(const TensorDesc* __restrict__ descs, const uint32_t* __rest
     int nvalid[kRowsPerWarp];
     bool vec[kRowsPerWarp];
     float amax[kRowsPerWarp];
-#pragma unroll
-    for (int k = 0; k < kRowsPerWarp; ++k) {
-        row_extent<GENERIC>(T, blk0 + k, lane, i0[k], nvalid[k], vec[k]);
-        const float s_old = (blk0 + k < T.n_blocks) ? load_scale(T.scale, blk0 + k, bf16_scale) : 1.0f;
-        amax[k] = lane_front<FMT, OPT>(T, P, i0[k], nvalid[k], vec[k], s_old, L[k], true);
-    }
-    const float my_amax = reduce_rows4(amax, lane);   // row (lane / 8)
-    float s_mine, inv_mine;
-    uint32_t bits_mine;
-    make_scale<FMT>(my_amax, bf16_scale, s_mine, inv_mine, bits_mine);
     const int g = lane >> 3;
-    if ((lane & 7) == 0 && blk0 + g < T.n_blocks) store_scale(T.scale, blk0 + g, bf16_scale, s_mine, bits_mine);
+    if constexpr (SUB == 4) {
 #pragma unroll
-    for (int k = 0; k < kRowsPerWarp; ++k) {
-        const float s = __shfl_sync(0xFFFFFFFFu, s_mine, 8 * k);
-        const float inv = __shfl_sync(0xFFFFFFFFu, inv_mine, 8 * k);
-        lane_back<FMT, OPT, RND>(T, P, i0[k], nvalid[k], vec[k], s, inv, L[k]);
+        for (int k = 0; k < kRowsPerWarp; ++k) {
+            row_extent<GENERIC>(T, blk0 + k, lane, i0[k], nvalid[k], vec[k]);
+            uint64_t sk;
+            const bool present = scale32_index<GENERIC>(T, blk0 + k, g, sk);
+            const float s_old = present ? load_scale(T.scale, sk, scale_kind) : 1.0f;
+            amax[k] = lane_front<FMT, OPT>(T, P, i0[k], nvalid[k], vec[k], s_old, L[k], true);
+        }
+#pragma unroll
+        for (int k = 0; k < kRowsPerWarp; ++k) {
+            float s, inv;
+            uint32_t bits;
+            make_scale<FMT>(group8_max(amax[k]), scale_kind, s, inv, bits);
+            uint64_t sk;
+            if (scale32_index<GENERIC>(T, blk0 + k, g, sk) && (lane & 7) == 0) store_scale(T.scale, sk, scale_kind, s, bits);
+            lane_back<FMT, OPT, RND>(T, P, i0[k], nvalid[k], vec[k], s, inv, L[k]);
+        }
+    } else {
+#pragma unroll
+        for (int k = 0; k < kRowsPerWarp; ++k) {
+            row_extent<GENERIC>(T, blk0 + k, lane, i0[k], nvalid[k], vec[k]);
+            const float s_old = (blk0 + k < T.n_blocks) ? load_scale(T.scale, blk0 + k, scale_kind) : 1.0f;
+            amax[k] = lane_front<FMT, OPT>(T, P, i0[k], nvalid[k], vec[k], s_old, L[k], true);
+        }
+        const float my_amax = reduce_rows4(amax, lane);   // row (lane / 8)
+        float s_mine, inv_mine;
+        uint32_t bits_mine;
+        make_scale<FMT>(my_amax, scale_kind, s_mine, inv_mine, bits_mine);
+        if ((lane & 7) == 0 && blk0 + g < T.n_blocks) store_scale(T.scale, blk0 + g, scale_kind, s_mine, bits_mine);
+#pragma unroll
+        for (int k = 0; k < kRowsPerWarp; ++k) {
+            const float s = __shfl_sync(0xFFFFFFFFu, s_mine, 8 * k);
+            const float inv = __shfl_sync(0xFFFFFFFFu, inv_mine, 8 * k);
+            lane_back<FMT, OPT, RND>(T, P, i0[k], nvalid[k], vec[k], s, inv, L[k]);
+        }
     }
 }
 
@@ -118,7 +159,7 @@ eco_block128_kernel(const TensorDesc* __restrict__ descs, const uint32_t* __rest
 template <int FMT, int OPT>
 __global__ void __launch_bounds__(kThreads)
 eco_tensor_amax_kernel(const TensorDesc* __restrict__ descs, const uint32_t* __restrict__ unit_tensor,
-                       const StepParams P, const int bf16_scale,
+                       const StepParams P, const int scale_kind,
                        uint32_t* __restrict__ scratch_amax, float* __restrict__ scratch_s_old) {
     __shared__ float smax[kWarps];
     const uint32_t unit = blockIdx.x;
@@ -126,7 +167,7 @@ eco_tensor_amax_kernel(const TensorDesc* __restrict__ descs, const uint32_t* __r
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t local = unit - T.first_unit;
     const uint64_t blk0 = static_cast<uint64_t>(local) * kRowsPerUnit + warp * kRowsPerWarp;
-    const float s_old = load_scale(T.scale, 0, bf16_scale);
+    const float s_old = load_scale(T.scale, 0, scale_kind);
     if (local == 0 && threadIdx.x == 0) scratch_s_old[T.slot] = s_old;
     float amax = 0.0f;
 #pragma unroll
@@ -153,7 +194,7 @@ eco_tensor_amax_kernel(const TensorDesc* __restrict__ descs, const uint32_t* __r
 template <int FMT, int OPT, int RND>
 __global__ void __launch_bounds__(kThreads)
 eco_tensor_apply_kernel(const TensorDesc* __restrict__ descs, const uint32_t* __restrict__ unit_tensor,
-                        const StepParams P, const int bf16_scale,
+                        const StepParams P, const int scale_kind,
                         const uint32_t* __restrict__ scratch_amax, uint32_t* __restrict__ scratch_amax_next,
                         const float* __restrict__ scratch_s_old, const int reverse, const uint32_t n_units) {
     const uint32_t unit = reverse ? (n_units - 1 - blockIdx.x) : blockIdx.x;
@@ -164,9 +205,9 @@ eco_tensor_apply_kernel(const TensorDesc* __restrict__ descs, const uint32_t* __
     const float s_old = scratch_s_old[T.slot];
     float s, inv;
     uint32_t s_bits;
-    make_scale<FMT>(__uint_as_float(scratch_amax[T.slot]), bf16_scale, s, inv, s_bits);
+    make_scale<FMT>(__uint_as_float(scratch_amax[T.slot]), scale_kind, s, inv, s_bits);
     if (local == 0 && threadIdx.x == 0) {
-        store_scale(T.scale, 0, bf16_scale, s, s_bits);
+        store_scale(T.scale, 0, scale_kind, s, s_bits);
         scratch_amax_next[T.slot] = 0u;
     }
 #pragma unroll
@@ -187,7 +228,7 @@ eco_tensor_apply_kernel(const TensorDesc* __restrict__ descs, const uint32_t* __
 template <int FMT, int OPT, int RND>
 __global__ void __launch_bounds__(kThreads)
 eco_row_kernel(const TensorDesc* __restrict__ descs, const uint32_t* __restrict__ unit_tensor,
-               const StepParams P, const int bf16_scale) {
+               const StepParams P, const int scale_kind) {
     __shared__ float smax[kWarps];
     __shared__ float s_sh, inv_sh;
     const uint32_t unit = blockIdx.x;
@@ -196,7 +237,7 @@ eco_row_kernel(const TensorDesc* __restrict__ descs, const uint32_t* __restrict_
     const uint64_t row = unit - T.first_unit;
     const uint64_t start = row * T.cols;
     const bool vec = (start & 3) == 0;
-    const float s_old = load_scale(T.scale, row, bf16_scale);
+    const float s_old = load_scale(T.scale, row, scale_kind);
     float amax = 0.0f;
     for (uint32_t c = 4 * threadIdx.x; c < T.cols; c += 4 * kThreads) {
         const uint32_t rem = T.cols - c;
@@ -212,8 +253,8 @@ eco_row_kernel(const TensorDesc* __restrict__ descs, const uint32_t* __restrict_
         for (int i = 1; i < kWarps; ++i) a = fmaxf(a, smax[i]);
         float s, inv;
         uint32_t s_bits;
-        make_scale<FMT>(a, bf16_scale, s, inv, s_bits);
-        store_scale(T.scale, row, bf16_scale, s, s_bits);
+        make_scale<FMT>(a, scale_kind, s, inv, s_bits);
+        store_scale(T.scale, row, scale_kind, s, s_bits);
         s_sh = s;
         inv_sh = inv;
     }
@@ -261,7 +302,7 @@ __device__ __forceinline__ float amax_lane(const float* x, uint64_t i0, int nval
 template <int FMT, int RND>
 __global__ void __launch_bounds__(kThreads)
 eco_quantize_kernel(const float* __restrict__ x, uint8_t* __restrict__ w, void* __restrict__ scale,
-                    const uint64_t rows, const uint32_t cols, const int mode, const int bf16_scale,
+                    const uint64_t rows, const uint32_t cols, const int mode, const int scale_kind,
                     const StepParams P, const uint32_t tensor_id, uint32_t* __restrict__ scratch_amax) {
     __shared__ float smax[kWarps];
     __shared__ float s_sh, inv_sh;
@@ -271,8 +312,8 @@ eco_quantize_kernel(const float* __restrict__ x, uint8_t* __restrict__ w, void* 
         float s = 0.f, inv = 0.f;
         uint32_t s_bits;
         if (mode == 1) {
-            make_scale<FMT>(__uint_as_float(*scratch_amax), bf16_scale, s, inv, s_bits);
-            if (blockIdx.x == 0 && threadIdx.x == 0) store_scale(scale, 0, bf16_scale, s, s_bits);
+            make_scale<FMT>(__uint_as_float(*scratch_amax), scale_kind, s, inv, s_bits);
+            if (blockIdx.x == 0 && threadIdx.x == 0) store_scale(scale, 0, scale_kind, s, s_bits);
         }
         float amax = 0.0f;
         for (uint64_t i0 = (static_cast<uint64_t>(blockIdx.x) * kThreads + threadIdx.x) * 4; i0 < numel;
@@ -303,8 +344,8 @@ eco_quantize_kernel(const float* __restrict__ x, uint8_t* __restrict__ w, void* 
                 for (int i = 1; i < kWarps; ++i) a = fmaxf(a, smax[i]);
                 float s, inv;
                 uint32_t s_bits;
-                make_scale<FMT>(a, bf16_scale, s, inv, s_bits);
-                store_scale(scale, row, bf16_scale, s, s_bits);
+                make_scale<FMT>(a, scale_kind, s, inv, s_bits);
+                store_scale(scale, row, scale_kind, s, s_bits);
                 s_sh = s;
                 inv_sh = inv;
             }
@@ -316,7 +357,7 @@ eco_quantize_kernel(const float* __restrict__ x, uint8_t* __restrict__ w, void* 
         }
         return;
     }
-    // mode 3: one warp per scale block
+    // mode 3 / 4: one warp per chunk of 128 elements of a row = one scale block (mode 3) or four of 32 (mode 4)
     const uint32_t bpr = (cols + 127u) / 128u;
     const uint64_t n_blocks = rows * bpr;
     for (uint64_t blk = static_cast<uint64_t>(blockIdx.x) * kWarps + warp; blk < n_blocks;
@@ -328,11 +369,18 @@ eco_quantize_kernel(const float* __restrict__ x, uint8_t* __restrict__ w, void* 
         const bool vec = (start & 3) == 0;
         const int rem = static_cast<int>(len) - 4 * lane;
         const int nvalid = rem < 0 ? 0 : (rem > 4 ? 4 : rem);
-        const float amax = warp_max(amax_lane(x, start + 4 * lane, nvalid, vec));
+        const float mine = amax_lane(x, start + 4 * lane, nvalid, vec);
         float s, inv;
         uint32_t s_bits;
-        make_scale<FMT>(amax, bf16_scale, s, inv, s_bits);
-        if (lane == 0) store_scale(scale, blk, bf16_scale, s, s_bits);
+        if (mode == 4) {
+            make_scale<FMT>(group8_max(mine), scale_kind, s, inv, s_bits);
+            const uint32_t g = static_cast<uint32_t>(lane) >> 3;
+            if ((lane & 7) == 0 && c0 + 32u * g < cols)
+                store_scale(scale, row * ((cols + 31u) / 32u) + c0 / 32u + g, scale_kind, s, s_bits);
+        } else {
+            make_scale<FMT>(warp_max(mine), scale_kind, s, inv, s_bits);
+            if (lane == 0) store_scale(scale, blk, scale_kind, s, s_bits);
+        }
         quantize_lane<FMT, RND>(x, w, start + 4 * lane, nvalid, vec, inv, P, tensor_id);
     }
 }
@@ -355,8 +403,13 @@ cudaError_t launch_block128(const LaunchConfig& c, const TensorDesc* descs, cons
                             uint32_t n_units, bool generic, const StepParams& P, cudaStream_t stream) {
     if (n_units == 0) return cudaSuccess;
     ECO_DISPATCH_FMT(c.format, ECO_DISPATCH_OPT(c.optimizer, ECO_DISPATCH_RND(c.rounding, {
-        if (generic) eco_block128_kernel<F, O, R, true><<<n_units, kThreads, 0, stream>>>(descs, unit_tensor, P, c.bf16_scale);
-        else eco_block128_kernel<F, O, R, false><<<n_units, kThreads, 0, stream>>>(descs, unit_tensor, P, c.bf16_scale);
+        if (c.sub == 4) {
+            if (generic) eco_block128_kernel<F, O, R, true, 4><<<n_units, kThreads, 0, stream>>>(descs, unit_tensor, P, c.scale_kind);
+            else eco_block128_kernel<F, O, R, false, 4><<<n_units, kThreads, 0, stream>>>(descs, unit_tensor, P, c.scale_kind);
+        } else {
+            if (generic) eco_block128_kernel<F, O, R, true, 1><<<n_units, kThreads, 0, stream>>>(descs, unit_tensor, P, c.scale_kind);
+            else eco_block128_kernel<F, O, R, false, 1><<<n_units, kThreads, 0, stream>>>(descs, unit_tensor, P, c.scale_kind);
+        }
     })))
     return cudaGetLastError();
 }
@@ -366,7 +419,7 @@ cudaError_t launch_tensor_amax(const LaunchConfig& c, const TensorDesc* descs, c
                                cudaStream_t stream) {
     if (n_units == 0) return cudaSuccess;
     ECO_DISPATCH_FMT(c.format, ECO_DISPATCH_OPT(c.optimizer, {
-        eco_tensor_amax_kernel<F, O><<<n_units, kThreads, 0, stream>>>(descs, unit_tensor, P, c.bf16_scale,
+        eco_tensor_amax_kernel<F, O><<<n_units, kThreads, 0, stream>>>(descs, unit_tensor, P, c.scale_kind,
                                                                      scratch_amax, scratch_s_old);
     }))
     return cudaGetLastError();
@@ -379,7 +432,7 @@ cudaError_t launch_tensor_apply(const LaunchConfig& c, const TensorDesc* descs, 
     if (n_units == 0) return cudaSuccess;
     ECO_DISPATCH_FMT(c.format, ECO_DISPATCH_OPT(c.optimizer, ECO_DISPATCH_RND(c.rounding, {
         eco_tensor_apply_kernel<F, O, R><<<n_units, kThreads, 0, stream>>>(
-            descs, unit_tensor, P, c.bf16_scale, scratch_amax, scratch_amax_next, scratch_s_old, reverse ? 1 : 0, n_units);
+            descs, unit_tensor, P, c.scale_kind, scratch_amax, scratch_amax_next, scratch_s_old, reverse ? 1 : 0, n_units);
     })))
     return cudaGetLastError();
 }
@@ -388,7 +441,7 @@ cudaError_t launch_row(const LaunchConfig& c, const TensorDesc* descs, const uin
                        uint32_t n_units, const StepParams& P, cudaStream_t stream) {
     if (n_units == 0) return cudaSuccess;
     ECO_DISPATCH_FMT(c.format, ECO_DISPATCH_OPT(c.optimizer, ECO_DISPATCH_RND(c.rounding, {
-        eco_row_kernel<F, O, R><<<n_units, kThreads, 0, stream>>>(descs, unit_tensor, P, c.bf16_scale);
+        eco_row_kernel<F, O, R><<<n_units, kThreads, 0, stream>>>(descs, unit_tensor, P, c.scale_kind);
     })))
     return cudaGetLastError();
 }
@@ -397,7 +450,7 @@ cudaError_t launch_quantize(const LaunchConfig& c, const float* x, uint8_t* w, v
                             uint32_t cols, int mode, const StepParams& P, uint32_t tensor_id,
                             uint32_t* scratch_amax, uint32_t grid, cudaStream_t stream) {
     ECO_DISPATCH_FMT(c.format, ECO_DISPATCH_RND(c.rounding, {
-        eco_quantize_kernel<F, R><<<grid, kThreads, 0, stream>>>(x, w, scale, rows, cols, mode, c.bf16_scale, P,
+        eco_quantize_kernel<F, R><<<grid, kThreads, 0, stream>>>(x, w, scale, rows, cols, mode, c.scale_kind, P,
                                                                 tensor_id, scratch_amax);
     }))
     return cudaGetLastError();
@@ -406,12 +459,12 @@ cudaError_t launch_quantize(const LaunchConfig& c, const float* x, uint8_t* w, v
 // ---------------------------------------------------------------------------
 // x^ = value(code) * scale (Sec. 3.1) for a whole tensor: what the forward pass of quantized training reads.
 // One thread per 4 consecutive elements of a row (cols is even for INT4, so a thread never splits a byte);
-// gran: 0 per-tensor, 1 per-row, 2 blocks of 128 along the row.  OUT_BF16: round the product to bf16 (nearest even).
+// gran: 0 per-tensor, 1 per-row, 2 blocks of `block` (128 or 32) elements along the row.  OUT_BF16: round the product to bf16 (nearest even).
 // ---------------------------------------------------------------------------
 template <int FMT, bool OUT_BF16>
 __global__ void __launch_bounds__(kThreads)
 eco_dequantize_kernel(const uint8_t* __restrict__ w, const void* __restrict__ scale, void* __restrict__ out,
-                      const uint64_t rows, const uint32_t cols, const int gran, const int bf16_scale) {
+                      const uint64_t rows, const uint32_t cols, const int gran, const uint32_t block, const int scale_kind) {
     const uint32_t quads_per_row = (cols + 3u) / 4u;
     const uint64_t n_quads = rows * quads_per_row;
     for (uint64_t qd = static_cast<uint64_t>(blockIdx.x) * kThreads + threadIdx.x; qd < n_quads;
@@ -427,8 +480,8 @@ eco_dequantize_kernel(const uint8_t* __restrict__ w, const void* __restrict__ sc
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
             if (e >= nvalid) break;
-            const uint64_t k = gran == 0 ? 0 : (gran == 1 ? row : row * ((cols + 127u) / 128u) + (c0 + e) / 128u);
-            const float x = __fmul_rn(val[e], load_scale(scale, k, bf16_scale));
+            const uint64_t k = gran == 0 ? 0 : (gran == 1 ? row : row * ((cols + block - 1u) / block) + (c0 + e) / block);
+            const float x = __fmul_rn(val[e], load_scale(scale, k, scale_kind));
             if (OUT_BF16) static_cast<uint16_t*>(out)[i0 + e] = static_cast<uint16_t>(f32_to_bf16_bits_rne(x));
             else static_cast<float*>(out)[i0 + e] = x;
         }
@@ -438,8 +491,8 @@ eco_dequantize_kernel(const uint8_t* __restrict__ w, const void* __restrict__ sc
 cudaError_t launch_dequantize(const LaunchConfig& c, const uint8_t* w, const void* scale, void* out, uint64_t rows,
                               uint32_t cols, int gran, bool out_bf16, uint32_t grid, cudaStream_t stream) {
     ECO_DISPATCH_FMT(c.format, {
-        if (out_bf16) eco_dequantize_kernel<F, true><<<grid, kThreads, 0, stream>>>(w, scale, out, rows, cols, gran, c.bf16_scale);
-        else eco_dequantize_kernel<F, false><<<grid, kThreads, 0, stream>>>(w, scale, out, rows, cols, gran, c.bf16_scale);
+        if (out_bf16) eco_dequantize_kernel<F, true><<<grid, kThreads, 0, stream>>>(w, scale, out, rows, cols, gran, static_cast<uint32_t>(128 / c.sub), c.scale_kind);
+        else eco_dequantize_kernel<F, false><<<grid, kThreads, 0, stream>>>(w, scale, out, rows, cols, gran, static_cast<uint32_t>(128 / c.sub), c.scale_kind);
     })
     return cudaGetLastError();
 }

@@ -13,7 +13,8 @@ struct LaunchConfig {
     int format;      // FMT_*
     int optimizer;   // OPT_*
     int rounding;    // RND_*
-    int bf16_scale;  // 0: f32 scales, 1: bf16 scales
+    int scale_kind;  // SCALE_KIND_*: f32, bf16 or power-of-two (one exponent byte) scales
+    int sub;         // block scales: scale blocks per 128 elements of a row (1: 1x128 blocks, 4: 1x32 blocks)
 };
 
 // Rows of 128 elements that one CTA (work unit) covers.
@@ -21,9 +22,9 @@ int rows_per_unit();
 int stream_unit_rows();
 
 // Modes of the TMA-fed streaming kernel (eco_stream_kernels.cu).
-enum : int { STREAM_BLOCK = 0, STREAM_TENSOR_AMAX = 1, STREAM_TENSOR_APPLY = 2, STREAM_ROW = 3 };
+enum : int { STREAM_BLOCK = 0, STREAM_TENSOR_AMAX = 1, STREAM_TENSOR_APPLY = 2, STREAM_ROW = 3, STREAM_BLOCK32 = 4 };
 enum : int { MODE_BLOCK = STREAM_BLOCK, MODE_TENSOR_AMAX = STREAM_TENSOR_AMAX, MODE_TENSOR_APPLY = STREAM_TENSOR_APPLY,
-             MODE_ROW = STREAM_ROW };
+             MODE_ROW = STREAM_ROW, MODE_BLOCK32 = STREAM_BLOCK32 };
 
 // Persistent launch over n_units work units; grid = min(n_units, grid_cap).  `tickets` are two device
 // words, zero before the first launch, that the kernel uses to hand out units and rewinds before it ends

@@ -54,8 +54,8 @@ template <int FMT, int OPT>
 struct StageLayout {
     static constexpr int kCodeRow = FMT == FMT_INT4 ? 64 : 128;  // bytes of codes per row
     static constexpr int kHeader = 0;
-    static constexpr int kScales = 128;                          // kUnitRows floats
-    static constexpr int kCodes = kScales + kUnitRows * 4;
+    static constexpr int kScales = 128;                          // up to 4 floats per row (blocks of 32 elements)
+    static constexpr int kCodes = kScales + kUnitRows * 16;
     static constexpr int kGrad = kCodes + kUnitRows * kCodeRow;
     static constexpr int kM = kGrad + kUnitRows * 256;
     static constexpr int kV = kM + kUnitRows * 512;
@@ -121,7 +121,7 @@ __device__ __forceinline__ uint32_t units_of(const TensorDesc& T) {
 // One unit (up to 32 rows of 128 elements) by the 8 consumer warps: warp w owns rows 4w..4w+3, lane l
 // elements 4l..4l+3 of each.  FULL: all 32 rows are present (every unit but the last of a tensor).
 template <int FMT, int OPT, int RND, int MODE, bool FULL, bool ERR, int NS = 4>
-__device__ __forceinline__ bool consume_unit(const StepParams& P, const int bf16_scale, const uint8_t* st,
+__device__ __forceinline__ bool consume_unit(const StepParams& P, const int scale_kind, const uint8_t* st,
                                              const StageHeader* h, const uint32_t empty_bar, const int warp,
                                              const int lane, uint32_t* scratch_amax, uint32_t& cur_slot,
                                              float& run_max, float* xchg, const uint32_t row_bars,
@@ -164,6 +164,7 @@ __device__ __forceinline__ bool consume_unit(const StepParams& P, const int bf16
                     v[k][0] = vr.x; v[k][1] = vr.y; v[k][2] = vr.z; v[k][3] = vr.w;
                 }
                 if (MODE == MODE_BLOCK) s_old = reinterpret_cast<const float*>(st + SL::kScales)[row];
+                else if (MODE == MODE_BLOCK32) s_old = reinterpret_cast<const float*>(st + SL::kScales)[row * 4 + (lane >> 3)];
                 else if (MODE == MODE_ROW) s_old = reinterpret_cast<const float*>(st + SL::kScales)[(row * h->div_magic) >> 16];
                 else s_old = h->s_old;
             }
@@ -220,13 +221,27 @@ __device__ __forceinline__ bool consume_unit(const StepParams& P, const int bf16
         const float my_amax = g8 == 0 ? rmax[0] : (g8 == 1 ? rmax[1] : (g8 == 2 ? rmax[2] : rmax[3]));
         float s_mine, inv_mine;
         uint32_t bits_mine;
-        make_scale<FMT>(my_amax, bf16_scale, s_mine, inv_mine, bits_mine);
+        make_scale<FMT>(my_amax, scale_kind, s_mine, inv_mine, bits_mine);
         if ((lane & 7) == 0 && (FULL || r + g8 < nrows))
-            store_scale(sp, row0 + r + g8, bf16_scale, s_mine, bits_mine);
+            store_scale(sp, row0 + r + g8, scale_kind, s_mine, bits_mine);
 #pragma unroll
         for (int k = 0; k < 4; ++k) {
             s_k[k] = __shfl_sync(0xFFFFFFFFu, s_mine, 8 * k);
             inv_k[k] = __shfl_sync(0xFFFFFFFFu, inv_mine, 8 * k);
+        }
+    } else if (MODE == MODE_BLOCK32) {
+        // four scale blocks of 32 elements per row: 8 lanes each; every lane derives the scale of its own block
+        const int g8 = lane >> 3;
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            float z = amax[k];
+            z = fmaxf(z, __shfl_xor_sync(0xFFFFFFFFu, z, 4));
+            z = fmaxf(z, __shfl_xor_sync(0xFFFFFFFFu, z, 2));
+            z = fmaxf(z, __shfl_xor_sync(0xFFFFFFFFu, z, 1));
+            uint32_t bits;
+            make_scale<FMT>(z, scale_kind, s_k[k], inv_k[k], bits);
+            if ((lane & 7) == 0 && (FULL || r + k < nrows))
+                store_scale(sp, (row0 + r + k) * 4 + g8, scale_kind, s_k[k], bits);
         }
     } else if (MODE == MODE_ROW) {
         // One scale per matrix row = seg_per_row consecutive 128-element rows, which belong to several warps.
@@ -249,11 +264,11 @@ __device__ __forceinline__ bool consume_unit(const StepParams& P, const int bf16
             const float a = warp_amax(x);
             float s_j, inv_j;
             uint32_t bits_j;
-            make_scale<FMT>(a, bf16_scale, s_j, inv_j, bits_j);
+            make_scale<FMT>(a, scale_kind, s_j, inv_j, bits_j);
             if (lane == 0) {
                 xs[j] = s_j;
                 xinv[j] = inv_j;
-                store_scale(sp, mrow0 + j, bf16_scale, s_j, bits_j);
+                store_scale(sp, mrow0 + j, scale_kind, s_j, bits_j);
             }
         }
         __syncwarp();
@@ -295,6 +310,7 @@ __device__ __forceinline__ bool consume_unit(const StepParams& P, const int bf16
 
 // ---------------------------------------------------------------------------
 // MODE_BLOCK        1x128 block scales, whole step in one pass
+// MODE_BLOCK32      1x32 block scales (four per 128-element row), whole step in one pass
 // MODE_TENSOR_AMAX  per-tensor scale, pass 1: max |theta~| per tensor
 // MODE_TENSOR_APPLY per-tensor scale, pass 2: quantize with the tensor's scale
 // MODE_ROW          one scale per matrix row of up to 32 * 128 columns, whole step in one pass; a unit is
@@ -309,7 +325,7 @@ template <int FMT, int OPT, int RND, int MODE, bool ERR>
 // register file, but the hardware was measured to place only one such CTA per SM.)
 __global__ void __launch_bounds__(kStreamThreads, 2)
 eco_stream_kernel(const TensorDesc* __restrict__ descs, const uint32_t* __restrict__ unit_tensor,
-                  const uint32_t n_units, const StepParams P, const int bf16_scale,
+                  const uint32_t n_units, const StepParams P, const int scale_kind,
                   uint32_t* __restrict__ scratch_amax, uint32_t* __restrict__ scratch_amax_next,
                   float* __restrict__ scratch_s_old, const int reverse, const int interleave,
                   uint32_t* __restrict__ tickets, uint32_t* __restrict__ status) {
@@ -386,24 +402,30 @@ eco_stream_kernel(const TensorDesc* __restrict__ descs, const uint32_t* __restri
                 h.seg_per_row = T.blocks_per_row; h.div_magic = 65536u / T.blocks_per_row + 1u;
                 h.n_mrows = n_mrows; h.pad_ = 0u; h.mrow0 = mrow0; h.index_base = T.index_base; h.e = T.e;
                 if (MODE == MODE_TENSOR_AMAX) {
-                    h.s_old = load_scale(T.scale, 0, bf16_scale);
+                    h.s_old = load_scale(T.scale, 0, scale_kind);
                     if (local == 0) scratch_s_old[T.slot] = h.s_old;
                 }
                 if (MODE == MODE_TENSOR_APPLY) {
                     h.s_old = scratch_s_old[T.slot];
                     uint32_t bits;
-                    make_scale<FMT>(__uint_as_float(scratch_amax[T.slot]), bf16_scale, h.s_new, h.inv_new, bits);
+                    make_scale<FMT>(__uint_as_float(scratch_amax[T.slot]), scale_kind, h.s_new, h.inv_new, bits);
                     if (local == 0) {
-                        store_scale(T.scale, 0, bf16_scale, h.s_new, bits);
+                        store_scale(T.scale, 0, scale_kind, h.s_new, bits);
                         scratch_amax_next[T.slot] = 0u;
                     }
                 }
                 *reinterpret_cast<StageHeader*>(st + SL::kHeader) = h;
             }
             if (MODE == MODE_BLOCK && lane < static_cast<int>(nrows))
-                reinterpret_cast<float*>(st + SL::kScales)[lane] = load_scale(T.scale, row0 + lane, bf16_scale);
+                reinterpret_cast<float*>(st + SL::kScales)[lane] = load_scale(T.scale, row0 + lane, scale_kind);
+            if (MODE == MODE_BLOCK32) {
+#pragma unroll
+                for (int j = 0; j < 4; ++j)
+                    if (lane * 4 + j < static_cast<int>(nrows) * 4)
+                        reinterpret_cast<float*>(st + SL::kScales)[lane * 4 + j] = load_scale(T.scale, row0 * 4 + lane * 4 + j, scale_kind);
+            }
             if (MODE == MODE_ROW && lane < static_cast<int>(n_mrows))
-                reinterpret_cast<float*>(st + SL::kScales)[lane] = load_scale(T.scale, mrow0 + lane, bf16_scale);
+                reinterpret_cast<float*>(st + SL::kScales)[lane] = load_scale(T.scale, mrow0 + lane, scale_kind);
             __syncwarp();
             if (lane == 0) mbar_arrive(full);
             ++it;
@@ -450,19 +472,19 @@ eco_stream_kernel(const TensorDesc* __restrict__ descs, const uint32_t* __restri
             // rows are dealt round-robin: this warp has rows warp, warp + 8, ... below nrows
             const int mine = static_cast<int>(nrows) > warp ? (static_cast<int>(nrows) - warp + kConsumerWarps - 1) / kConsumerWarps : 0;
             if (mine == 4)
-                ok = consume_unit<FMT, OPT, RND, MODE, true, ERR, 4>(P, bf16_scale, st, h, empty, warp, lane, scratch_amax, cur_slot,
+                ok = consume_unit<FMT, OPT, RND, MODE, true, ERR, 4>(P, scale_kind, st, h, empty, warp, lane, scratch_amax, cur_slot,
                                                                      run_max, xchg, row_bars, it & 1u, status);
             else if (mine == 3)
-                ok = consume_unit<FMT, OPT, RND, MODE, true, ERR, 3>(P, bf16_scale, st, h, empty, warp, lane, scratch_amax, cur_slot,
+                ok = consume_unit<FMT, OPT, RND, MODE, true, ERR, 3>(P, scale_kind, st, h, empty, warp, lane, scratch_amax, cur_slot,
                                                                      run_max, xchg, row_bars, it & 1u, status);
             else
-                ok = consume_unit<FMT, OPT, RND, MODE, false, ERR, 4>(P, bf16_scale, st, h, empty, warp, lane, scratch_amax, cur_slot,
+                ok = consume_unit<FMT, OPT, RND, MODE, false, ERR, 4>(P, scale_kind, st, h, empty, warp, lane, scratch_amax, cur_slot,
                                                                       run_max, xchg, row_bars, it & 1u, status);
         } else if (nrows == kUnitRows)   // (discarded statement of the if constexpr above for the per-row mode)
-            ok = consume_unit<FMT, OPT, RND, MODE, true, ERR>(P, bf16_scale, st, h, empty, warp, lane, scratch_amax, cur_slot,
+            ok = consume_unit<FMT, OPT, RND, MODE, true, ERR>(P, scale_kind, st, h, empty, warp, lane, scratch_amax, cur_slot,
                                                               run_max, xchg, row_bars, it & 1u, status);
         else
-            ok = consume_unit<FMT, OPT, RND, MODE, false, ERR>(P, bf16_scale, st, h, empty, warp, lane, scratch_amax, cur_slot,
+            ok = consume_unit<FMT, OPT, RND, MODE, false, ERR>(P, scale_kind, st, h, empty, warp, lane, scratch_amax, cur_slot,
                                                                run_max, xchg, row_bars, it & 1u, status);
         if (!ok) return;
     }
@@ -475,7 +497,7 @@ eco_stream_kernel(const TensorDesc* __restrict__ descs, const uint32_t* __restri
 // ---------------------------------------------------------------------------
 template <int FMT, int OPT, int RND, int MODE, bool ERR = false>
 static cudaError_t launch_one(const TensorDesc* descs, const uint32_t* unit_tensor, uint32_t n_units, const StepParams& P,
-                              int bf16_scale, uint32_t* amax, uint32_t* amax_next, float* s_old, bool reverse,
+                              int scale_kind, uint32_t* amax, uint32_t* amax_next, float* s_old, bool reverse,
                               uint32_t* tickets, uint32_t* status, int grid_cap, cudaStream_t stream) {
     using SL = StageLayout<FMT, OPT>;
     static bool configured = false;
@@ -486,9 +508,9 @@ static cudaError_t launch_one(const TensorDesc* descs, const uint32_t* unit_tens
         configured = true;
     }
     const uint32_t grid = n_units < static_cast<uint32_t>(grid_cap) ? n_units : static_cast<uint32_t>(grid_cap);
-    kernel<<<grid, kStreamThreads, SL::kSmem, stream>>>(descs, unit_tensor, n_units, P, bf16_scale, amax, amax_next,
+    kernel<<<grid, kStreamThreads, SL::kSmem, stream>>>(descs, unit_tensor, n_units, P, scale_kind, amax, amax_next,
                                                         s_old, reverse ? 1 : 0,
-                                                        (MODE == MODE_BLOCK || MODE == MODE_ROW) ? kInterleave : 1, tickets, status);
+                                                        (MODE == MODE_BLOCK || MODE == MODE_BLOCK32 || MODE == MODE_ROW) ? kInterleave : 1, tickets, status);
     return cudaGetLastError();
 }
 
@@ -510,21 +532,23 @@ cudaError_t launch_stream(const LaunchConfig& c, int mode, const TensorDesc* des
     if (n_units == 0) return cudaSuccess;
     if (mode == STREAM_TENSOR_AMAX) {
         ECO_S_FMT(c.format, ECO_S_OPT(c.optimizer, {
-            return launch_one<F, O, RND_RTN, MODE_TENSOR_AMAX>(descs, unit_tensor, n_units, P, c.bf16_scale, amax,
+            return launch_one<F, O, RND_RTN, MODE_TENSOR_AMAX>(descs, unit_tensor, n_units, P, c.scale_kind, amax,
                                                                amax_next, s_old, reverse, tickets, status, grid_cap, stream);
         }))
     }
 #define ECO_S_LAUNCH(MODE_, ERR_)                                                                                      \
-    return launch_one<F, O, R, MODE_, ERR_>(descs, unit_tensor, n_units, P, c.bf16_scale, amax, amax_next, s_old, reverse, \
+    return launch_one<F, O, R, MODE_, ERR_>(descs, unit_tensor, n_units, P, c.scale_kind, amax, amax_next, s_old, reverse, \
                                             tickets, status, grid_cap, stream)
     ECO_S_FMT(c.format, ECO_S_OPT(c.optimizer, ECO_S_RND(c.rounding, {
         if (with_errors) {
             if (mode == STREAM_ROW) ECO_S_LAUNCH(MODE_ROW, true);
             if (mode == STREAM_BLOCK) ECO_S_LAUNCH(MODE_BLOCK, true);
+            if (mode == STREAM_BLOCK32) ECO_S_LAUNCH(MODE_BLOCK32, true);
             ECO_S_LAUNCH(MODE_TENSOR_APPLY, true);
         }
         if (mode == STREAM_ROW) ECO_S_LAUNCH(MODE_ROW, false);
         if (mode == STREAM_BLOCK) ECO_S_LAUNCH(MODE_BLOCK, false);
+        if (mode == STREAM_BLOCK32) ECO_S_LAUNCH(MODE_BLOCK32, false);
         ECO_S_LAUNCH(MODE_TENSOR_APPLY, false);
     })))
 #undef ECO_S_LAUNCH

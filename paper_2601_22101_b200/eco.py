@@ -19,7 +19,7 @@ ECO_OK = 0
 ECO_ERR_INVALID_ARG, ECO_ERR_UNSUPPORTED, ECO_ERR_ALIGNMENT, ECO_ERR_CUDA, ECO_ERR_NOMEM, ECO_ERR_TIMEOUT = 1, 2, 3, 4, 5, 6
 ECO_FORMAT_FP8_E4M3, ECO_FORMAT_INT4, ECO_FORMAT_FP8_E5M2 = 0, 1, 4
 ECO_SCALE_PER_TENSOR, ECO_SCALE_PER_ROW, ECO_SCALE_PER_BLOCK = 0, 1, 2
-ECO_SCALE_F32, ECO_SCALE_BF16 = 0, 1
+ECO_SCALE_F32, ECO_SCALE_BF16, ECO_SCALE_E8M0 = 0, 1, 2
 ECO_OPT_SGDM, ECO_OPT_ADAM = 0, 1
 ECO_ROUND_NEAREST, ECO_ROUND_STOCHASTIC = 0, 1
 ECO_INJECT_NONE, ECO_INJECT_ECO, ECO_INJECT_EXACT = 0, 1, 2

@@ -42,7 +42,7 @@ class DeviceState:
         dev = torch.device("cuda", device)
         ts = w.tensors
         adam = w.optimizer == wl.ADAM
-        sb = 4 if w.scale_dtype == wl.SCALE_F32 else 2
+        sb = wl.SCALE_BYTES[w.scale_dtype]
         self._w_off, w_total = _carve([w.code_bytes(t) for t in ts])
         self._s_off, s_total = _carve([w.n_scales(t) * sb for t in ts])
         self._g_off, g_total = _carve([t.numel * 2 for t in ts])
@@ -53,7 +53,7 @@ class DeviceState:
         self.m_buf = torch.zeros(m_total, dtype=torch.uint8, device=dev)
         self.v_buf = torch.zeros(m_total, dtype=torch.uint8, device=dev) if adam else None
         self.tensors: List[eco.Tensor] = []
-        sdt = torch.float32 if w.scale_dtype == wl.SCALE_F32 else torch.bfloat16
+        sdt = {wl.SCALE_F32: torch.float32, wl.SCALE_BF16: torch.bfloat16, wl.SCALE_E8M0: torch.uint8}[w.scale_dtype]
         for i, t in enumerate(ts):
             cw = self.w_buf[self._w_off[i]: self._w_off[i] + w.code_bytes(t)]
             cs = self.s_buf[self._s_off[i]: self._s_off[i] + w.n_scales(t) * sb].view(sdt)

@@ -22,7 +22,8 @@ import numpy as np
 # Enumerations of the C-ABI (include/eco.h), by value.
 FP8_E4M3, INT4, FP8_E5M2 = 0, 1, 4
 PER_TENSOR, PER_ROW, PER_BLOCK = 0, 1, 2
-SCALE_F32, SCALE_BF16 = 0, 1
+SCALE_F32, SCALE_BF16, SCALE_E8M0 = 0, 1, 2
+SCALE_BYTES = {SCALE_F32: 4, SCALE_BF16: 2, SCALE_E8M0: 1}
 SGDM, ADAM = 0, 1
 RTN, SR = 0, 1
 
@@ -87,7 +88,7 @@ class Workload:
         w = 0.5 if self.format == INT4 else 1.0
         moments = 4.0 * (2 if self.optimizer == ADAM else 1)
         n_scale = sum(self.n_scales(t) for t in self.tensors)
-        sb = (4.0 if self.scale_dtype == SCALE_F32 else 2.0) * n_scale / max(self.numel, 1)
+        sb = float(SCALE_BYTES[self.scale_dtype]) * n_scale / max(self.numel, 1)
         return (w + 2.0 + moments + sb) + (w + moments + sb)
 
 

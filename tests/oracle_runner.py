@@ -14,7 +14,8 @@ from paper_2601_22101_b200 import workloads as wl
 def oracle_config(w: wl.Workload, injection: int = oracle.INJECT_ECO) -> oracle.Config:
     # the enumerations of the boundary and of the oracle agree by value
     return oracle.Config(format=w.format, granularity=w.granularity, block=w.block,
-                         scale_dtype=oracle.SCALE_BF16 if w.scale_dtype == wl.SCALE_BF16 else oracle.SCALE_NATIVE,
+                         scale_dtype={wl.SCALE_F32: oracle.SCALE_NATIVE, wl.SCALE_BF16: oracle.SCALE_BF16,
+                                      wl.SCALE_E8M0: oracle.SCALE_E8M0}[w.scale_dtype],
                          optimizer=w.optimizer, rounding=w.rounding, injection=injection,
                          grad_dtype=oracle.GRAD_BF16)
 

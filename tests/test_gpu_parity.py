@@ -20,10 +20,14 @@ def _np(t):
 
 def _scale_bits(t):
     t = t.detach().cpu()
+    if t.dtype == torch.uint8:
+        return t.numpy().astype(np.int32)
     return (t.view(torch.int16) if t.dtype == torch.bfloat16 else t.view(torch.int32)).numpy()
 
 
 def _oracle_scale_bits(s):
+    if s.dtype == np.uint8:
+        return s.astype(np.int32)
     return s.view(np.int16) if s.dtype == np.uint16 else s.view(np.int32)
 
 
@@ -62,9 +66,9 @@ def run_chained(w: wl.Workload, steps: int, check_every: int = 1, injection=eco.
     return dev, ora
 
 
-def _mini(fmt, gran, sdt, opt, rnd, shapes, lr=1e-3, grad_std=1e-3):
+def _mini(fmt, gran, sdt, opt, rnd, shapes, lr=1e-3, grad_std=1e-3, block=128):
     ts = [wl.TensorSpec(f"t{i}", r, c, 100 + 7 * i, zero_grad=(i == 1 and len(shapes) > 2)) for i, (r, c) in enumerate(shapes)]
-    return wl.Workload("mini", fmt, gran, 128, sdt, opt, rnd, lr=lr, beta1=0.9, beta2=0.95, eps=1e-8,
+    return wl.Workload("mini", fmt, gran, block, sdt, opt, rnd, lr=lr, beta1=0.9, beta2=0.95, eps=1e-8,
                        weight_std=0.02, grad_std=grad_std, steps=6, step_seed=0xABCDEF0123, tensors=ts)
 
 
@@ -518,5 +522,53 @@ def test_e5m2_step_and_quantize_parity(rnd, opt, gran):
         eco.eco_dequantize(config_of(w), dw, ds, t.rows, t.cols, out)
         torch.cuda.synchronize()
         assert (_np(dw) == ow).all() and (_np(ds).view(np.int32) == os_.view(np.int32)).all()
+        ref = oracle.dequantize(oracle_config(w), ow, os_, t.rows, t.cols)
+        assert (_np(out).view(np.int32) == ref.reshape(-1).view(np.int32)).all()
+
+
+MX_SHAPES = RAGGED + RAGGED_FP8_ONLY + [(40, 512), (3, 75), (2, 4128)]
+
+
+@pytest.mark.parametrize("opt", [wl.SGDM, wl.ADAM])
+@pytest.mark.parametrize("rnd", [wl.RTN, wl.SR])
+@pytest.mark.parametrize("fmt,sdt,block", [(wl.FP8_E4M3, wl.SCALE_E8M0, 32), (wl.FP8_E5M2, wl.SCALE_E8M0, 32),
+                                           (wl.INT4, wl.SCALE_E8M0, 32), (wl.FP8_E4M3, wl.SCALE_F32, 32),
+                                           (wl.INT4, wl.SCALE_BF16, 32), (wl.FP8_E4M3, wl.SCALE_E8M0, 128)])
+def test_blocks_of_32_and_power_of_two_scales(fmt, sdt, block, rnd, opt):
+    """1x32 scale blocks (streaming kernel for whole 128-element rows, direct-load kernel for ragged ones) and
+    power-of-two scales stored as one exponent byte, chained steps against the oracle."""
+    shapes = [s_ for s_ in MX_SHAPES if fmt != wl.INT4 or s_[1] % 2 == 0]
+    run_chained(_mini(fmt, wl.PER_BLOCK, sdt, opt, rnd, shapes, block=block), steps=5)
+
+
+@pytest.mark.parametrize("gran", [wl.PER_TENSOR, wl.PER_ROW])
+def test_power_of_two_scales_with_tensor_and_row_granularity(gran):
+    run_chained(_mini(wl.FP8_E4M3, gran, wl.SCALE_E8M0, wl.ADAM, wl.SR, RAGGED + RAGGED_FP8_ONLY), steps=4)
+
+
+@pytest.mark.parametrize("fmt,sdt", [(wl.FP8_E4M3, wl.SCALE_E8M0), (wl.INT4, wl.SCALE_E8M0), (wl.FP8_E5M2, wl.SCALE_F32)])
+@pytest.mark.parametrize("rnd", [wl.RTN, wl.SR])
+def test_quantize_and_dequantize_blocks_of_32(fmt, sdt, rnd):
+    rng = np.random.default_rng(23)
+    shapes = [s_ for s_ in MX_SHAPES if fmt != wl.INT4 or s_[1] % 2 == 0]
+    w = _mini(fmt, wl.PER_BLOCK, sdt, wl.SGDM, rnd, shapes, block=32)
+    sdt_t = {wl.SCALE_F32: torch.float32, wl.SCALE_E8M0: torch.uint8}[sdt]
+    for t in w.tensors:
+        x = (rng.standard_normal((t.rows, t.cols)) * 0.02).astype(np.float32)
+        x.flat[:: 17] = 0.0
+        x.flat[:: 29] *= 1e-4
+        if t.cols >= 64:
+            x[0, :32] = 0.0                                  # an all-zero block
+            if sdt == wl.SCALE_E8M0:
+                x[-1, 32:64] *= np.float32(1e-38)            # a block whose scale clamps at the smallest exponent
+        ow, os_ = oracle.quantize(oracle_config(w), x, seed=5, step=9, tensor_id=t.tensor_id)
+        dw = torch.zeros(w.code_bytes(t), dtype=torch.uint8, device="cuda")
+        ds = torch.zeros(w.n_scales(t), dtype=sdt_t, device="cuda")
+        eco.eco_quantize(config_of(w), torch.from_numpy(x).cuda(), t.rows, t.cols, dw, ds, seed=5, step=9, tensor_id=t.tensor_id)
+        out = torch.zeros(t.numel, dtype=torch.float32, device="cuda")
+        eco.eco_dequantize(config_of(w), dw, ds, t.rows, t.cols, out)
+        torch.cuda.synchronize()
+        assert (_np(dw) == ow).all(), (t.rows, t.cols)
+        assert (_scale_bits(ds) == _oracle_scale_bits(os_)).all(), (t.rows, t.cols)
         ref = oracle.dequantize(oracle_config(w), ow, os_, t.rows, t.cols)
         assert (_np(out).view(np.int32) == ref.reshape(-1).view(np.int32)).all()
