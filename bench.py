@@ -53,7 +53,7 @@ def _dominant_kernel(w) -> str:
     fmt = {wl.FP8_E4M3: "fp8", wl.INT4: "int4", wl.FP8_E5M2: "e5m2"}[w.format]
     opt = "adam" if w.optimizer == wl.ADAM else "sgdm"
     rnd = "sr" if w.rounding == wl.SR else "rtn"
-    mode = {wl.PER_BLOCK: "block", wl.PER_TENSOR: "tensor_apply", wl.PER_ROW: "row"}[w.granularity]
+    mode = {wl.PER_BLOCK: "block" if w.block == 128 else "block32", wl.PER_TENSOR: "tensor_apply", wl.PER_ROW: "row"}[w.granularity]
     return f"eco_stream_kernel<{fmt},{opt},{rnd},{mode}>"
 
 
@@ -253,7 +253,7 @@ def main():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=5)
-    ap.add_argument("--workload", default="c4", choices=["c1", "c2", "c3", "c4", "c5", "c3r", "c5t", "c4g", "c4d", "c3s", "c3rs", "c4s", "c5s"])
+    ap.add_argument("--workload", default="c4", choices=["c1", "c2", "c3", "c4", "c5", "c3r", "c5t", "c4g", "c4d", "c3s", "c3rs", "c4s", "c5s", "c4mx", "c4mxs", "c4ds"])
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--also", default="c3,c5", help="comma-separated workloads timed after the headline one and "
                     "reported under other_workloads (device-resident timing only)")

@@ -296,7 +296,9 @@ eco_status eco_create(eco_ctx** out, const eco_config* cfg, const eco_tensor* te
     ctx->lc = launch_config(*cfg);
     ctx->reverse_pass2 = g_options.reverse_pass2 != 0;
     ctx->grid_cap = static_cast<int>(g_options.ctas_per_sm) * prop.multiProcessorCount;
-    const bool use_stream = g_options.use_stream != 0;
+    // the streaming kernels take 1x32 blocks with power-of-two scales (the microscaling layout) and every other
+    // granularity with f32 / bf16 scales; the remaining combinations run on the direct-load kernels
+    const bool use_stream = g_options.use_stream != 0 && ((ctx->lc.scale_kind == eco::SCALE_KIND_E8M0) == (ctx->lc.sub == 4));
 
     ctx->desc_of_tensor.assign(n, 0);
     // ---- work-unit tables -------------------------------------------------

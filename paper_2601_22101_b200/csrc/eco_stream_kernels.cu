@@ -221,7 +221,7 @@ __device__ __forceinline__ bool consume_unit(const StepParams& P, const int scal
         const float my_amax = g8 == 0 ? rmax[0] : (g8 == 1 ? rmax[1] : (g8 == 2 ? rmax[2] : rmax[3]));
         float s_mine, inv_mine;
         uint32_t bits_mine;
-        make_scale<FMT>(my_amax, scale_kind, s_mine, inv_mine, bits_mine);
+        make_scale_div<FMT>(my_amax, scale_kind == SCALE_KIND_BF16, s_mine, inv_mine, bits_mine);
         if ((lane & 7) == 0 && (FULL || r + g8 < nrows))
             store_scale(sp, row0 + r + g8, scale_kind, s_mine, bits_mine);
 #pragma unroll
@@ -230,18 +230,25 @@ __device__ __forceinline__ bool consume_unit(const StepParams& P, const int scal
             inv_k[k] = __shfl_sync(0xFFFFFFFFu, inv_mine, 8 * k);
         }
     } else if (MODE == MODE_BLOCK32) {
-        // four scale blocks of 32 elements per row: 8 lanes each; every lane derives the scale of its own block
-        const int g8 = lane >> 3;
+        // Four scale blocks of 32 elements per row, 8 lanes each: 16 maxima per warp.  Three butterfly stages inside
+        // each group of 8 lanes, halving the number of rows a lane carries at each: afterwards lane l holds the
+        // maximum of row (l >> 1) & 3 over its group.  It derives that one scale; the four scales a lane needs come
+        // back from lanes 0, 2, 4, 6 of its group.
+        const bool b2 = lane & 4, b1 = lane & 2;
+        const float x = fmaxf(b2 ? amax[2] : amax[0], __shfl_xor_sync(0xFFFFFFFFu, b2 ? amax[0] : amax[2], 4));
+        const float y = fmaxf(b2 ? amax[3] : amax[1], __shfl_xor_sync(0xFFFFFFFFu, b2 ? amax[1] : amax[3], 4));
+        float z = fmaxf(b1 ? y : x, __shfl_xor_sync(0xFFFFFFFFu, b1 ? x : y, 2));
+        z = fmaxf(z, __shfl_xor_sync(0xFFFFFFFFu, z, 1));
+        const int rr = (lane >> 1) & 3, g8 = lane >> 3;
+        float s_mine, inv_mine;
+        uint32_t bits_mine;
+        make_scale_pow2<FMT>(z, s_mine, inv_mine, bits_mine);
+        if ((lane & 1) == 0 && (FULL || r + rr < nrows))
+            static_cast<uint8_t*>(sp)[(row0 + r + rr) * 4 + g8] = static_cast<uint8_t>(bits_mine);
 #pragma unroll
         for (int k = 0; k < 4; ++k) {
-            float z = amax[k];
-            z = fmaxf(z, __shfl_xor_sync(0xFFFFFFFFu, z, 4));
-            z = fmaxf(z, __shfl_xor_sync(0xFFFFFFFFu, z, 2));
-            z = fmaxf(z, __shfl_xor_sync(0xFFFFFFFFu, z, 1));
-            uint32_t bits;
-            make_scale<FMT>(z, scale_kind, s_k[k], inv_k[k], bits);
-            if ((lane & 7) == 0 && (FULL || r + k < nrows))
-                store_scale(sp, (row0 + r + k) * 4 + g8, scale_kind, s_k[k], bits);
+            s_k[k] = __shfl_sync(0xFFFFFFFFu, s_mine, (lane & 24) + 2 * k);
+            inv_k[k] = __shfl_sync(0xFFFFFFFFu, inv_mine, (lane & 24) + 2 * k);
         }
     } else if (MODE == MODE_ROW) {
         // One scale per matrix row = seg_per_row consecutive 128-element rows, which belong to several warps.
@@ -264,7 +271,7 @@ __device__ __forceinline__ bool consume_unit(const StepParams& P, const int scal
             const float a = warp_amax(x);
             float s_j, inv_j;
             uint32_t bits_j;
-            make_scale<FMT>(a, scale_kind, s_j, inv_j, bits_j);
+            make_scale_div<FMT>(a, scale_kind == SCALE_KIND_BF16, s_j, inv_j, bits_j);
             if (lane == 0) {
                 xs[j] = s_j;
                 xinv[j] = inv_j;
@@ -310,13 +317,14 @@ __device__ __forceinline__ bool consume_unit(const StepParams& P, const int scal
 
 // ---------------------------------------------------------------------------
 // MODE_BLOCK        1x128 block scales, whole step in one pass
-// MODE_BLOCK32      1x32 block scales (four per 128-element row), whole step in one pass
+// MODE_BLOCK32      1x32 blocks (four per 128-element row) with power-of-two scales, whole step in one pass
 // MODE_TENSOR_AMAX  per-tensor scale, pass 1: max |theta~| per tensor
 // MODE_TENSOR_APPLY per-tensor scale, pass 2: quantize with the tensor's scale
 // MODE_ROW          one scale per matrix row of up to 32 * 128 columns, whole step in one pass; a unit is
 //                   floor(32 / R) whole matrix rows of R 128-element rows each
 // Tensors handled here have a whole number of 128-element rows that start on
 // 128-element boundaries (cols % 128 == 0, or a flat tensor with numel % 128 == 0).
+// MODE_BLOCK32 takes power-of-two scales only; the other modes take f32 and bf16 scales only.
 // ---------------------------------------------------------------------------
 // ERR: the tensors carry error buffers (see eco_attach_error_buffers); a separate instantiation, so that the plain
 // method pays nothing for the option.
@@ -408,7 +416,7 @@ eco_stream_kernel(const TensorDesc* __restrict__ descs, const uint32_t* __restri
                 if (MODE == MODE_TENSOR_APPLY) {
                     h.s_old = scratch_s_old[T.slot];
                     uint32_t bits;
-                    make_scale<FMT>(__uint_as_float(scratch_amax[T.slot]), scale_kind, h.s_new, h.inv_new, bits);
+                    make_scale_div<FMT>(__uint_as_float(scratch_amax[T.slot]), scale_kind == SCALE_KIND_BF16, h.s_new, h.inv_new, bits);
                     if (local == 0) {
                         store_scale(T.scale, 0, scale_kind, h.s_new, bits);
                         scratch_amax_next[T.slot] = 0u;
@@ -422,7 +430,7 @@ eco_stream_kernel(const TensorDesc* __restrict__ descs, const uint32_t* __restri
 #pragma unroll
                 for (int j = 0; j < 4; ++j)
                     if (lane * 4 + j < static_cast<int>(nrows) * 4)
-                        reinterpret_cast<float*>(st + SL::kScales)[lane * 4 + j] = load_scale(T.scale, row0 * 4 + lane * 4 + j, scale_kind);
+                        reinterpret_cast<float*>(st + SL::kScales)[lane * 4 + j] = load_scale(T.scale, row0 * 4 + lane * 4 + j, SCALE_KIND_E8M0);
             }
             if (MODE == MODE_ROW && lane < static_cast<int>(n_mrows))
                 reinterpret_cast<float*>(st + SL::kScales)[lane] = load_scale(T.scale, mrow0 + lane, scale_kind);

@@ -268,8 +268,29 @@ def c4_dense() -> Workload:
     return replace(w, name="c4_smoe_2mat_fp8_block128_adam_sr_all_routed", tensors=[replace(t, zero_grad=False) for t in w.tensors])
 
 
+def c4_mx() -> Workload:
+    """The all-routed sparse-MoE set in the microscaling layout: FP8-E4M3 codes, 1x32 blocks, one power-of-two
+    exponent byte per block (20.03 B/param)."""
+    w = c4_dense()
+    return replace(w, name="c4_smoe_2mat_mxfp8_block32_e8m0_adam_sr_all_routed", block=32, scale_dtype=SCALE_E8M0)
+
+
+def c4_mx_small() -> Workload:
+    """c4_mx cut to the size of c4_small (profiling-sized)."""
+    w = c4_small()
+    return replace(w, name="c4_smoe_2mat_mxfp8_block32_e8m0_adam_sr_small", block=32, scale_dtype=SCALE_E8M0,
+                   tensors=[replace(t, zero_grad=False) for t in w.tensors])
+
+
+def c4_dense_small() -> Workload:
+    """c4_dense cut to the size of c4_small (profiling-sized)."""
+    w = c4_small()
+    return replace(w, name="c4_smoe_2mat_fp8_block128_adam_sr_all_routed_small", tensors=[replace(t, zero_grad=False) for t in w.tensors])
+
+
 BY_NAME = {"c1": c1, "c2": c2, "c3": c3, "c4": c4, "c5": c5, "c3r": c3_rowwise, "c5t": c5_tensorwise_adam, "c4g": lambda: c4(expert_mats=3), "c4d": c4_dense,
-           "c3s": c3_small, "c3rs": c3_rowwise_small, "c4s": c4_small, "c5s": c5_small}
+           "c3s": c3_small, "c3rs": c3_rowwise_small, "c4s": c4_small, "c5s": c5_small,
+           "c4mx": c4_mx, "c4mxs": c4_mx_small, "c4ds": c4_dense_small}
 
 
 def _rng(w: Workload, t: TensorSpec, step: int, kind: int) -> np.random.Generator:
