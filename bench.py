@@ -37,7 +37,9 @@ NCU_DRAM_BYTES_PER_PARAM = {
     # profiles/eco_stream_kernel_c5s.md: 1.1941 GB + 0.7723 GB over 183,304,192 parameters
     "eco_stream_kernel<int4,sgdm,sr,block>": 10.73,
     # profiles/eco_stream_kernel_c3s.md (apply pass): 1.0058 GB + 0.7672 GB over 91,422,720 parameters
-    "eco_stream_kernel<fp8,adam,sr,tensor_apply>": 19.42,
+    "eco_stream_kernel<fp8,adam,sr,tensor_apply>": 19.41,
+    # profiles/eco_stream_kernel_c4mxs.md: 1.4808 GB + 1.1617 GB over 134,217,728 parameters
+    "eco_stream_kernel<fp8,adam,sr,block32>": 19.69,
 }
 
 
@@ -255,7 +257,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--workload", default="c4", choices=["c1", "c2", "c3", "c4", "c5", "c3r", "c5t", "c4g", "c4d", "c3s", "c3rs", "c4s", "c5s", "c4mx", "c4mxs", "c4ds"])
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--also", default="c3,c5", help="comma-separated workloads timed after the headline one and "
+    ap.add_argument("--also", default="c3,c5,c4mx", help="comma-separated workloads timed after the headline one and "
                     "reported under other_workloads (device-resident timing only)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
