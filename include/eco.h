@@ -132,7 +132,12 @@ eco_status eco_create(eco_ctx** out, const eco_config* cfg, const eco_tensor* te
  * Asynchronous: enqueues its kernels on cuda_stream and returns; it never
  * synchronizes and never allocates.  Consecutive steps of one context must be
  * ordered on the device (same stream, or events), because they share the
- * context's reduction scratch.
+ * context's reduction scratch.  The call can be recorded by a stream capture
+ * (CUDA graph); a replay repeats the recorded step index, seed and
+ * hyper-parameters.  With ECO_SCALE_PER_TENSOR the reduction scratch alternates
+ * between two halves from one call to the next (each call clears the half the
+ * next one accumulates into), so a graph for that granularity must hold an even
+ * number of consecutive eco_step calls.
  * Errors: ECO_ERR_INVALID_ARG for lr <= 0 or non-finite (alpha = (1/lr)(..) is
  * undefined, Eq. 7), beta1 outside (0,1) (1/beta1), Adam beta2 outside (0,1),
  * eps < 0, step < 1; ECO_ERR_CUDA for a failed launch.  On ECO_ERR_INVALID_ARG

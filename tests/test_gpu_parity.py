@@ -279,7 +279,8 @@ def _sampled_full_size(w: wl.Workload, sample_ids, steps=2):
     before = {}
     for i in sample_ids:
         d = dev.tensors[i]
-        before[i] = [d.w.cpu().numpy().copy(), _np(d.scale.view(torch.int16 if d.scale.dtype == torch.bfloat16 else torch.float32)).copy(),
+        sview = {torch.bfloat16: torch.int16, torch.uint8: torch.uint8}.get(d.scale.dtype, torch.float32)
+        before[i] = [d.w.cpu().numpy().copy(), _np(d.scale.view(sview)).copy(),
                      d.grad.view(torch.int16).cpu().numpy().view(np.uint16).copy(), d.m.cpu().numpy().copy(),
                      None if d.v is None else d.v.cpu().numpy().copy()]
         if w.scale_dtype == wl.SCALE_BF16:
@@ -317,6 +318,13 @@ def test_c4_full_size_sampled_tensors():
     ids = set(_spread(len(w.tensors), 24))
     ids |= set([i for i, t in enumerate(w.tensors) if t.zero_grad][:: 200])      # make sure zero-gradient experts are in
     _sampled_full_size(w, sorted(ids))
+
+
+def test_c4_microscaling_full_size_sampled_tensors():
+    """The all-routed sparse-MoE set in the microscaling layout (1x32 blocks, power-of-two scales), as the benchmark
+    times it."""
+    w = wl.c4_mx()
+    _sampled_full_size(w, _spread(len(w.tensors), 16))
 
 
 def test_c3_full_size_sampled_tensors():
@@ -572,3 +580,34 @@ def test_quantize_and_dequantize_blocks_of_32(fmt, sdt, rnd):
         assert (_scale_bits(ds) == _oracle_scale_bits(os_)).all(), (t.rows, t.cols)
         ref = oracle.dequantize(oracle_config(w), ow, os_, t.rows, t.cols)
         assert (_np(out).view(np.int32) == ref.reshape(-1).view(np.int32)).all()
+
+
+def test_step_is_capturable_in_a_cuda_graph():
+    """eco_step neither allocates nor synchronises, so a stream capture records it; replaying the graph runs the
+    recorded step (same step index and seed) again on the current state.  Checked against the oracle taking the
+    same step index twice."""
+    w = _mini(wl.FP8_E4M3, wl.PER_BLOCK, wl.SCALE_F32, wl.ADAM, wl.SR, [(64, 256), (3, 384), (5, 200)])
+    dev = DeviceState(w)
+    dev.init_from_host()
+    ora = OracleState(w)
+    dev.create()
+    try:
+        grads = [wl.gradient_bf16(w, t, 1) for t in w.tensors]
+        for i, g in enumerate(grads):
+            dev.tensors[i].grad.view(torch.int16).copy_(torch.from_numpy(g.view(np.int16)))
+        torch.cuda.synchronize()
+        side = torch.cuda.Stream()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=side):
+            dev.step(1, stream=torch.cuda.current_stream().cuda_stream)
+        torch.cuda.synchronize()
+        compare_before = [_np(t.w).copy() for t in dev.tensors]
+        ora_before = [c.copy() for c in ora.w]
+        assert all((a == b).all() for a, b in zip(compare_before, ora_before)), "capture must not run the step"
+        for _ in range(2):
+            graph.replay()
+            ora.step(1, grads)
+        torch.cuda.synchronize()
+        compare(dev, ora, "after two replays")
+    finally:
+        dev.destroy()
