@@ -187,6 +187,7 @@ StepParams derive_params(const eco_config& cfg, float lr_f, float beta1_f, float
     P.beta1 = beta1_f;
     P.beta2 = beta2_f;
     P.eps = eps_f;
+    P.neg_eps = -eps_f;
     P.one_minus_beta1 = static_cast<float>(1.0 - b1);
     P.one_minus_beta2 = static_cast<float>(1.0 - b2);
     P.neg_lr = -lr_f;
@@ -201,6 +202,8 @@ StepParams derive_params(const eco_config& cfg, float lr_f, float beta1_f, float
         const double bc2 = 1.0 - std::pow(b2, t);
         P.inv_bc2 = static_cast<float>(1.0 / bc2);
         P.lr_over_bc1 = static_cast<float>(lr / bc1);
+        P.neg_lr_over_bc1 = -P.lr_over_bc1;
+        P.neg_inv_bc2 = -P.inv_bc2;
         P.adam_coef = static_cast<float>((bc1 / lr) * (1.0 - 1.0 / b1));
     }
     P.seed_lo = static_cast<uint32_t>(seed);
