@@ -329,7 +329,8 @@ eco_status eco_dequantize(const eco_config* cfg, const void* w, const void* scal
  *   "use_stream"      1 (default) uses the persistent kernels fed by bulk asynchronous copies
  *                     wherever a tensor consists of whole, aligned 128-element rows; 0 forces
  *                     the direct-load kernels everywhere
- *   "ctas_per_sm"     persistent grid size in CTAs per SM, 1 or 2 (default 2)
+ *   "ctas_per_sm"     persistent grid size in CTAs per SM, 1..3; 0 (default) = as many as the kernel is built to
+ *                     keep resident (3 for momentum SGD, 2 for Adam)
  * No option changes any result bit.  Errors: ECO_ERR_INVALID_ARG for an unknown name.
  */
 eco_status eco_set_option(const char* name, int64_t value);

@@ -38,7 +38,7 @@ struct Options {
     int64_t l2_group_bytes = 0;    // per-tensor scale: input bytes per launch pair; -1 = half of the L2 size, 0 = one group
     int64_t reverse_pass2 = 1;     // per-tensor scale: walk pass 2 in the opposite order of pass 1
     int64_t use_stream = 1;        // 1: TMA-fed persistent kernels where the layout allows; 0: direct-load kernels only
-    int64_t ctas_per_sm = 2;       // persistent grid = ctas_per_sm * SM count
+    int64_t ctas_per_sm = 0;       // persistent grid = ctas_per_sm * SM count; 0: the kernel's own residency (2 or 3)
 };
 Options g_options;
 
@@ -115,6 +115,7 @@ eco_status check_config(const eco_config* cfg, bool need_optimizer) {
 
 LaunchConfig launch_config(const eco_config& cfg) {
     LaunchConfig lc;
+    lc.sm_count = 0;
     lc.format = cfg.format == ECO_FORMAT_FP8_E4M3 ? eco::FMT_FP8 : (cfg.format == ECO_FORMAT_FP8_E5M2 ? eco::FMT_E5M2 : eco::FMT_INT4);
     lc.optimizer = cfg.optimizer == ECO_OPT_ADAM ? eco::OPT_ADAM : eco::OPT_SGDM;
     lc.rounding = cfg.rounding == ECO_ROUND_STOCHASTIC ? eco::RND_SR : eco::RND_RTN;
@@ -240,7 +241,7 @@ eco_status eco_set_option(const char* name, int64_t value) {
     if (!std::strcmp(name, "reverse_pass2")) { g_options.reverse_pass2 = value; return ECO_OK; }
     if (!std::strcmp(name, "use_stream")) { g_options.use_stream = value; return ECO_OK; }
     if (!std::strcmp(name, "ctas_per_sm")) {
-        if (value < 1 || value > 2) return fail(nullptr, ECO_ERR_INVALID_ARG, "ctas_per_sm must be 1 or 2");
+        if (value < 0 || value > 3) return fail(nullptr, ECO_ERR_INVALID_ARG, "ctas_per_sm must be 0 (automatic), 1, 2 or 3");
         g_options.ctas_per_sm = value;
         return ECO_OK;
     }
@@ -299,6 +300,7 @@ eco_status eco_create(eco_ctx** out, const eco_config* cfg, const eco_tensor* te
     ctx->lc = launch_config(*cfg);
     ctx->reverse_pass2 = g_options.reverse_pass2 != 0;
     ctx->grid_cap = static_cast<int>(g_options.ctas_per_sm) * prop.multiProcessorCount;
+    ctx->lc.sm_count = prop.multiProcessorCount;
     // the streaming kernels take 1x32 blocks with power-of-two scales (the microscaling layout) and every other
     // granularity with f32 / bf16 scales; the remaining combinations run on the direct-load kernels
     const bool use_stream = g_options.use_stream != 0 && ((ctx->lc.scale_kind == eco::SCALE_KIND_E8M0) == (ctx->lc.sub == 4));

@@ -14,6 +14,7 @@ struct LaunchConfig {
     int optimizer;   // OPT_*
     int rounding;    // RND_*
     int scale_kind;  // SCALE_KIND_*: f32, bf16 or power-of-two (one exponent byte) scales
+    int sm_count;    // SMs of the device (sizes the persistent grids)
     int sub;         // block scales: scale blocks per 128 elements of a row (1: 1x128 blocks, 4: 1x32 blocks)
 };
 
@@ -26,7 +27,8 @@ enum : int { STREAM_BLOCK = 0, STREAM_TENSOR_AMAX = 1, STREAM_TENSOR_APPLY = 2, 
 enum : int { MODE_BLOCK = STREAM_BLOCK, MODE_TENSOR_AMAX = STREAM_TENSOR_AMAX, MODE_TENSOR_APPLY = STREAM_TENSOR_APPLY,
              MODE_ROW = STREAM_ROW, MODE_BLOCK32 = STREAM_BLOCK32 };
 
-// Persistent launch over n_units work units; grid = min(n_units, grid_cap).  `tickets` are two device
+// Persistent launch over n_units work units; grid = min(n_units, grid_cap), where grid_cap = 0 stands for the kernel's
+// own number of resident CTAs per SM (3 for momentum SGD, 2 for Adam) times LaunchConfig::sm_count.  `tickets` are two device
 // words, zero before the first launch, that the kernel uses to hand out units and rewinds before it ends
 // (launches sharing them must be ordered on the device).  `status` is a device word that receives a
 // non-zero code if a bounded wait inside the kernel expires.  with_errors selects the instantiation that also

@@ -1,7 +1,7 @@
 // Streaming kernels of the ECO step for sm_100a: persistent CTAs fed by the TMA
 // engine.
 //
-// One CTA = 1 producer warp + 8 consumer warps, two CTAs per SM.  The parameter
+// One CTA = 1 producer warp + 8 consumer warps, two (Adam) or three (momentum SGD) CTAs per SM.  The parameter
 // set is cut into units of 32 rows of 128 elements (4096 parameters); each CTA
 // owns a contiguous range of units.  For every unit the producer issues one
 // bulk asynchronous copy (cp.async.bulk, global -> shared, completion counted
@@ -50,6 +50,10 @@ struct StageHeader {
 };
 static_assert(sizeof(StageHeader) <= 128, "header must fit its slot");
 
+// Resident CTAs per SM a kernel instantiation is compiled for (register budget 65536 / (288 * n)).
+template <int OPT, bool ERR>
+__host__ __device__ constexpr int stream_ctas_per_sm() { return (OPT == OPT_SGDM && !ERR) ? 3 : 2; }
+
 template <int FMT, int OPT>
 struct StageLayout {
     static constexpr int kCodeRow = FMT == FMT_INT4 ? 64 : 128;  // bytes of codes per row
@@ -60,7 +64,7 @@ struct StageLayout {
     static constexpr int kM = kGrad + kUnitRows * 256;
     static constexpr int kV = kM + kUnitRows * 512;
     static constexpr int kBytes = kV + (OPT == OPT_ADAM ? kUnitRows * 512 : 0);
-    static constexpr int kStages = OPT == OPT_ADAM ? 2 : 3;
+    static constexpr int kStages = 2;                            // x 2 (Adam) or 3 (SGDM) resident CTAs per SM
     static constexpr int kBarriers = 512;                        // 2 * kStages + 2 mbarriers, padded to 128; then the
                                                                  // per-row exchange: 32 maxima, 32 scales, 32 inverses
     static constexpr int kRowBars = 64;                          // two mbarriers of the per-row exchange
@@ -329,9 +333,11 @@ __device__ __forceinline__ bool consume_unit(const StepParams& P, const int scal
 // ERR: the tensors carry error buffers (see eco_attach_error_buffers); a separate instantiation, so that the plain
 // method pays nothing for the option.
 template <int FMT, int OPT, int RND, int MODE, bool ERR>
-// Two CTAs per SM: the compiler then allows 96 registers per thread.  (112 would still add up to less than the
-// register file, but the hardware was measured to place only one such CTA per SM.)
-__global__ void __launch_bounds__(kStreamThreads, 2)
+// Adam: two CTAs per SM, so the compiler allows 96 registers per thread.  (112 would still add up to less than the
+// register file, but the hardware was measured to place only one such CTA per SM.)  Momentum SGD carries no second
+// moment and fits 72 registers without spilling: three CTAs per SM, i.e. 24 consumer warps to hide the latencies of
+// its instruction-heavier bytes.
+__global__ void __launch_bounds__(kStreamThreads, stream_ctas_per_sm<OPT, ERR>())
 eco_stream_kernel(const TensorDesc* __restrict__ descs, const uint32_t* __restrict__ unit_tensor,
                   const uint32_t n_units, const StepParams P, const int scale_kind,
                   uint32_t* __restrict__ scratch_amax, uint32_t* __restrict__ scratch_amax_next,
@@ -506,7 +512,7 @@ eco_stream_kernel(const TensorDesc* __restrict__ descs, const uint32_t* __restri
 template <int FMT, int OPT, int RND, int MODE, bool ERR = false>
 static cudaError_t launch_one(const TensorDesc* descs, const uint32_t* unit_tensor, uint32_t n_units, const StepParams& P,
                               int scale_kind, uint32_t* amax, uint32_t* amax_next, float* s_old, bool reverse,
-                              uint32_t* tickets, uint32_t* status, int grid_cap, cudaStream_t stream) {
+                              uint32_t* tickets, uint32_t* status, int grid_cap, int sm_count, cudaStream_t stream) {
     using SL = StageLayout<FMT, OPT>;
     static bool configured = false;
     auto kernel = eco_stream_kernel<FMT, OPT, RND, MODE, ERR>;
@@ -515,7 +521,8 @@ static cudaError_t launch_one(const TensorDesc* descs, const uint32_t* unit_tens
         if (e != cudaSuccess) return e;
         configured = true;
     }
-    const uint32_t grid = n_units < static_cast<uint32_t>(grid_cap) ? n_units : static_cast<uint32_t>(grid_cap);
+    const uint32_t cap = static_cast<uint32_t>(grid_cap > 0 ? grid_cap : sm_count * stream_ctas_per_sm<OPT, ERR>());
+    const uint32_t grid = n_units < cap ? n_units : cap;
     kernel<<<grid, kStreamThreads, SL::kSmem, stream>>>(descs, unit_tensor, n_units, P, scale_kind, amax, amax_next,
                                                         s_old, reverse ? 1 : 0,
                                                         (MODE == MODE_BLOCK || MODE == MODE_BLOCK32 || MODE == MODE_ROW) ? kInterleave : 1, tickets, status);
@@ -541,12 +548,12 @@ cudaError_t launch_stream(const LaunchConfig& c, int mode, const TensorDesc* des
     if (mode == STREAM_TENSOR_AMAX) {
         ECO_S_FMT(c.format, ECO_S_OPT(c.optimizer, {
             return launch_one<F, O, RND_RTN, MODE_TENSOR_AMAX>(descs, unit_tensor, n_units, P, c.scale_kind, amax,
-                                                               amax_next, s_old, reverse, tickets, status, grid_cap, stream);
+                                                               amax_next, s_old, reverse, tickets, status, grid_cap, c.sm_count, stream);
         }))
     }
 #define ECO_S_LAUNCH(MODE_, ERR_)                                                                                      \
     return launch_one<F, O, R, MODE_, ERR_>(descs, unit_tensor, n_units, P, c.scale_kind, amax, amax_next, s_old, reverse, \
-                                            tickets, status, grid_cap, stream)
+                                            tickets, status, grid_cap, c.sm_count, stream)
     ECO_S_FMT(c.format, ECO_S_OPT(c.optimizer, ECO_S_RND(c.rounding, {
         if (with_errors) {
             if (mode == STREAM_ROW) ECO_S_LAUNCH(MODE_ROW, true);
