@@ -34,8 +34,8 @@ FALLBACK_HBM_GBS = 6650.0
 NCU_DRAM_BYTES_PER_PARAM = {
     # profiles/eco_stream_kernel_c4s.md: 1.4808 GB read + 1.1625 GB written over 134,217,728 parameters
     "eco_stream_kernel<fp8,adam,sr,block>": 19.69,
-    # profiles/eco_stream_kernel_c5s.md: 1.1941 GB + 0.7717 GB over 183,304,192 parameters
-    "eco_stream_kernel<int4,sgdm,sr,block>": 10.72,
+    # profiles/eco_stream_kernel_c5s.md: 1.1941 GB + 0.7726 GB over 183,304,192 parameters
+    "eco_stream_kernel<int4,sgdm,sr,block>": 10.73,
     # profiles/eco_stream_kernel_c3s.md (apply pass): 1.0058 GB + 0.7683 GB over 91,422,720 parameters
     "eco_stream_kernel<fp8,adam,sr,tensor_apply>": 19.41,
     # profiles/eco_stream_kernel_c4mxs.md: 1.4812 GB + 1.1603 GB over 134,217,728 parameters
