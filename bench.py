@@ -225,18 +225,37 @@ def run_e2e(w, device: int, steps: int, max_host_gb: float):
         total += t.numel
     ws = replace(w, tensors=picked)
     sdt = {wl.SCALE_F32: torch.float32, wl.SCALE_BF16: torch.bfloat16, wl.SCALE_E8M0: torch.uint8}[w.scale_dtype]
+    # the state lives in one pinned host buffer per kind (codes, scales, gradients, m, v), tensors back to back, as an
+    # offloaded optimizer keeps it; eco_host_step then moves each kind of a chunk in one copy
+    sb = wl.SCALE_BYTES[w.scale_dtype]
+    n_code = sum(ws.code_bytes(t) for t in ws.tensors)
+    n_scale = sum(ws.n_scales(t) for t in ws.tensors)
+    flat_w = torch.empty(n_code, dtype=torch.uint8, pin_memory=True).random_(0, 120)
+    flat_s = torch.empty(n_scale * sb, dtype=torch.uint8, pin_memory=True)
+    flat_g = torch.empty(total, dtype=torch.bfloat16, pin_memory=True)
+    flat_m = torch.zeros(total, dtype=torch.float32, pin_memory=True)
+    flat_v = torch.zeros(total, dtype=torch.float32, pin_memory=True) if adam else None
+    if w.scale_dtype == wl.SCALE_E8M0:
+        flat_s.fill_(114)                               # 2^-13
+    else:
+        flat_s.view(sdt).fill_(1e-4)
     tensors = []
+    ow = os_ = oe = 0
     for t in ws.tensors:
-        cw = torch.zeros(ws.code_bytes(t), dtype=torch.uint8).pin_memory()
-        cs = torch.ones(ws.n_scales(t), dtype=sdt).mul_(1e-4).pin_memory()
-        cw.random_(0, 120)
-        cg = torch.randn(t.numel, dtype=torch.float32).mul_(w.grad_std).to(torch.bfloat16).pin_memory()
-        cm = torch.zeros(t.numel, dtype=torch.float32).pin_memory()
-        cv = torch.zeros(t.numel, dtype=torch.float32).pin_memory() if adam else None
+        cw = flat_w[ow: ow + ws.code_bytes(t)]
+        cs = flat_s[os_: os_ + ws.n_scales(t) * sb].view(sdt)
+        cg = flat_g[oe: oe + t.numel]
+        cg.copy_(torch.randn(t.numel, dtype=torch.float32).mul_(w.grad_std).to(torch.bfloat16))
+        cm = flat_m[oe: oe + t.numel]
+        cv = flat_v[oe: oe + t.numel] if adam else None
         tensors.append(eco.Tensor(cw, cs, cg, cm, cv, t.rows, t.cols, t.tensor_id))
+        ow += ws.code_bytes(t)
+        os_ += ws.n_scales(t) * sb
+        oe += t.numel
     cfg = config_of(ws)
     up = down = 0
     handle = eco.eco_host_create(cfg, tensors, device)
+    n_in, n_out = eco.eco_host_copies(handle)
     eco.eco_host_step(handle, w.lr, w.beta1, w.beta2, w.eps, 1, w.step_seed)   # warm-up
     torch.cuda.synchronize(device)
     t0 = time.perf_counter()
@@ -246,6 +265,7 @@ def run_e2e(w, device: int, steps: int, max_host_gb: float):
     el = time.perf_counter() - t0
     eco.eco_host_destroy(handle)
     return {"value": ws.numel * steps / el, "unit": UNIT, "h2d_bytes_per_step": up, "d2h_bytes_per_step": down,
+            "h2d_copies_per_step": n_in, "d2h_copies_per_step": n_out,
             "steps": steps, "params_per_step": ws.numel, "seconds": el,
             "sample": f"first {len(picked)} of {len(w.tensors)} tensors per GPU held in pinned host memory"}
 

@@ -202,12 +202,19 @@ eco_status eco_step_end(eco_ctx* ctx, void* cuda_stream);
  *                    and the device-side status of every chunk has been checked.  h2d_bytes / d2h_bytes
  *                    (host, optional) receive the bytes copied in each direction.  The gradient buffers
  *                    are read at every call.  Errors: as eco_step, plus ECO_ERR_TIMEOUT.
+ *                    Inside a chunk the staging slot is laid out by kind (all codes, all scales, ...), and
+ *                    buffers that follow one another directly in ONE host allocation (a flat pinned buffer
+ *                    per kind, tensors back to back, sizes that are multiples of 256 bytes) travel in a single
+ *                    copy; anything else is copied buffer by buffer.
+ *   eco_host_copies  (host, optional outputs) the number of copies one eco_host_step issues in each
+ *                    direction; ECO_ERR_INVALID_ARG for a NULL context.
  *   eco_host_destroy frees all of it (synchronizes the device).  NULL is allowed.
  * eco_step_host is the one-shot form: create, one step, destroy.
  */
 eco_status eco_host_create(eco_host_ctx** out, const eco_config* cfg, const eco_tensor* tensors, size_t n, int device);
 eco_status eco_host_step(eco_host_ctx* ctx, float lr, float beta1, float beta2, float eps, uint64_t step, uint64_t seed,
                          uint64_t* h2d_bytes, uint64_t* d2h_bytes);
+eco_status eco_host_copies(const eco_host_ctx* ctx, uint64_t* h2d_copies, uint64_t* d2h_copies);
 eco_status eco_host_destroy(eco_host_ctx* ctx);
 eco_status eco_step_host(const eco_config* cfg, const eco_tensor* tensors, size_t n, int device,
                          float lr, float beta1, float beta2, float eps, uint64_t step, uint64_t seed,

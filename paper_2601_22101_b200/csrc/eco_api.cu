@@ -663,12 +663,14 @@ eco_status eco_quantize(const eco_config* cfg, const float* x, int64_t rows, int
 struct eco_host_ctx {
     struct Place { uint64_t w, scale, grad, m, v, wb, sb, gb, mb; };
     struct Chunk { size_t first, count; uint64_t bytes; };
+    struct Copy { void* dev; void* host; uint64_t bytes; };   // one cudaMemcpyAsync (several tensors when both sides are contiguous)
     eco_config cfg;
     int device = 0;
     bool adam = false;
     std::vector<eco_tensor> host, dev;
     std::vector<Place> place;
     std::vector<Chunk> chunks;
+    std::vector<std::vector<Copy>> copies_in, copies_out;   // per chunk
     std::vector<eco_ctx*> ctxs;
     std::vector<cudaEvent_t> ev_in, ev_run, ev_out;
     cudaStream_t s_in = nullptr, s_run = nullptr, s_out = nullptr;
@@ -676,6 +678,26 @@ struct eco_host_ctx {
     uint64_t slot_bytes = 0, up = 0, down = 0;
     int n_slots = 0;
 };
+
+// True when a and b lie inside the same CUDA allocation (pinned host memory or device memory): the driver reports
+// the start of the allocation a pointer belongs to.  Anything it does not know (pageable memory) is "no".
+static bool same_allocation(const void* a, const void* b) {
+    using Fn = int (*)(void*, int, unsigned long long);       // cuPointerGetAttribute(data, attribute, pointer)
+    static Fn fn = []() -> Fn {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuPointerGetAttribute", &p, cudaEnableDefault, &q) != cudaSuccess ||
+            q != cudaDriverEntryPointSuccess)
+            return nullptr;
+        return reinterpret_cast<Fn>(p);
+    }();
+    if (!fn) return false;
+    constexpr int kRangeStart = 11;                             // CU_POINTER_ATTRIBUTE_RANGE_START_ADDR
+    unsigned long long sa = 0, sb = 0;
+    if (fn(&sa, kRangeStart, reinterpret_cast<unsigned long long>(a)) != 0) return false;
+    if (fn(&sb, kRangeStart, reinterpret_cast<unsigned long long>(b)) != 0) return false;
+    return sa != 0 && sa == sb;
+}
 
 extern "C" {
 
@@ -717,6 +739,7 @@ eco_status eco_host_create(eco_host_ctx** out, const eco_config* cfg, const eco_
     constexpr uint64_t kChunkTarget = 256ull << 20;
     constexpr int kSlots = 3;
     {
+        // chunks: consecutive tensors up to the target size
         eco_host_ctx::Chunk c{0, 0, 0};
         for (size_t i = 0; i < n; ++i) {
             const uint64_t numel = static_cast<uint64_t>(tensors[i].rows) * static_cast<uint64_t>(tensors[i].cols);
@@ -728,22 +751,38 @@ eco_status eco_host_create(eco_host_ctx** out, const eco_config* cfg, const eco_
                 h->chunks.push_back(c);
                 c = eco_host_ctx::Chunk{i, 0, 0};
             }
-            uint64_t off = c.bytes;
-            p.w = off; off += align(p.wb);
-            p.scale = off; off += align(p.sb);
-            p.grad = off; off += align(p.gb);
-            p.m = off; off += align(p.mb);
-            p.v = off; if (adam) off += align(p.mb);
-            c.bytes = off;
+            c.bytes += need;
             c.count++;
             h->slot_bytes = std::max(h->slot_bytes, c.bytes);
         }
         h->chunks.push_back(c);
+        // inside a chunk the buffers are laid out by kind (all codes, all scales, all gradients, all m, all v), so
+        // that state which is contiguous on the host is contiguous on the device too and moves in one copy
+        for (const eco_host_ctx::Chunk& ch : h->chunks) {
+            uint64_t region[5] = {0, 0, 0, 0, 0};
+            for (size_t i = ch.first; i < ch.first + ch.count; ++i) {
+                const eco_host_ctx::Place& p = h->place[i];
+                region[0] += align(p.wb); region[1] += align(p.sb); region[2] += align(p.gb); region[3] += align(p.mb);
+                if (adam) region[4] += align(p.mb);
+            }
+            uint64_t off[5] = {0, region[0], region[0] + region[1], region[0] + region[1] + region[2],
+                               region[0] + region[1] + region[2] + region[3]};
+            for (size_t i = ch.first; i < ch.first + ch.count; ++i) {
+                eco_host_ctx::Place& p = h->place[i];
+                p.w = off[0]; off[0] += align(p.wb);
+                p.scale = off[1]; off[1] += align(p.sb);
+                p.grad = off[2]; off[2] += align(p.gb);
+                p.m = off[3]; off[3] += align(p.mb);
+                p.v = off[4]; if (adam) off[4] += align(p.mb);
+            }
+        }
     }
     h->n_slots = static_cast<int>(std::min<size_t>(kSlots, h->chunks.size()));
     const size_t nc = h->chunks.size();
     h->ctxs.assign(nc, nullptr);
     h->ev_in.assign(nc, nullptr); h->ev_run.assign(nc, nullptr); h->ev_out.assign(nc, nullptr);
+    h->copies_in.assign(nc, {});
+    h->copies_out.assign(nc, {});
 #define ECO_CUDA_H(call)                                                                             \
     do {                                                                                             \
         cudaError_t e_ = (call);                                                                     \
@@ -770,6 +809,28 @@ eco_status eco_host_create(eco_host_ctx** out, const eco_config* cfg, const eco_
         }
         eco_status rc = eco_create(&h->ctxs[c], cfg, h->dev.data() + h->chunks[c].first, h->chunks[c].count, device);
         if (rc != ECO_OK) { eco_host_destroy(h); return rc; }
+        // copy lists, kind by kind; a buffer joins the previous copy when it follows it directly on both sides and
+        // the two host buffers are parts of one allocation (neighbouring addresses alone do not make one copy legal)
+        auto add = [](std::vector<eco_host_ctx::Copy>& v, void* dev, const void* host, uint64_t bytes) {
+            if (!v.empty() && static_cast<uint8_t*>(v.back().dev) + v.back().bytes == dev &&
+                static_cast<uint8_t*>(v.back().host) + v.back().bytes == host && same_allocation(v.back().host, host))
+                v.back().bytes += bytes;
+            else
+                v.push_back(eco_host_ctx::Copy{dev, const_cast<void*>(host), bytes});
+        };
+        const size_t first = h->chunks[c].first, last = first + h->chunks[c].count;
+        for (int kind = 0; kind < 5; ++kind) {
+            if (kind == 4 && !adam) continue;
+            for (size_t i = first; i < last; ++i) {
+                const eco_host_ctx::Place& p = h->place[i];
+                const eco_tensor &hs = h->host[i], &dv = h->dev[i];
+                void* d = kind == 0 ? dv.w : kind == 1 ? dv.scale : kind == 2 ? const_cast<void*>(dv.grad) : kind == 3 ? static_cast<void*>(dv.m) : static_cast<void*>(dv.v);
+                const void* s = kind == 0 ? hs.w : kind == 1 ? hs.scale : kind == 2 ? hs.grad : kind == 3 ? static_cast<const void*>(hs.m) : static_cast<const void*>(hs.v);
+                const uint64_t b = kind == 0 ? p.wb : kind == 1 ? p.sb : kind == 2 ? p.gb : p.mb;
+                add(h->copies_in[c], d, s, b);
+                if (kind != 2) add(h->copies_out[c], d, s, b);      // the gradient is an input only
+            }
+        }
         ECO_CUDA_H(cudaEventCreateWithFlags(&h->ev_in[c], cudaEventDisableTiming));
         ECO_CUDA_H(cudaEventCreateWithFlags(&h->ev_run[c], cudaEventDisableTiming));
         ECO_CUDA_H(cudaEventCreateWithFlags(&h->ev_out[c], cudaEventDisableTiming));
@@ -779,26 +840,28 @@ eco_status eco_host_create(eco_host_ctx** out, const eco_config* cfg, const eco_
     return ECO_OK;
 }
 
+eco_status eco_host_copies(const eco_host_ctx* h, uint64_t* h2d_copies, uint64_t* d2h_copies) {
+    if (!h) return fail(nullptr, ECO_ERR_INVALID_ARG, "ctx is NULL");
+    uint64_t in = 0, out = 0;
+    for (const auto& v : h->copies_in) in += v.size();
+    for (const auto& v : h->copies_out) out += v.size();
+    if (h2d_copies) *h2d_copies = in;
+    if (d2h_copies) *d2h_copies = out;
+    return ECO_OK;
+}
+
 eco_status eco_host_step(eco_host_ctx* h, float lr, float beta1, float beta2, float eps, uint64_t step, uint64_t seed,
                          uint64_t* h2d_bytes, uint64_t* d2h_bytes) {
     if (!h) return fail(nullptr, ECO_ERR_INVALID_ARG, "ctx is NULL");
     if (eco_status st = check_hyper(nullptr, h->cfg, lr, beta1, beta2, eps, step)) return st;
     ECO_CUDA(nullptr, cudaSetDevice(h->device));
-    const bool adam = h->adam;
     uint64_t up = 0, down = 0;
     for (size_t c = 0; c < h->chunks.size(); ++c) {
-        const size_t first = h->chunks[c].first, last = first + h->chunks[c].count;
         // the slot is free once the chunk that used it before has been copied out
         if (c >= static_cast<size_t>(h->n_slots)) ECO_CUDA(nullptr, cudaStreamWaitEvent(h->s_in, h->ev_out[c - h->n_slots], 0));
-        for (size_t i = first; i < last; ++i) {
-            const eco_host_ctx::Place& p = h->place[i];
-            const eco_tensor &src = h->host[i], &dst = h->dev[i];
-            ECO_CUDA(nullptr, cudaMemcpyAsync(dst.w, src.w, p.wb, cudaMemcpyHostToDevice, h->s_in));
-            ECO_CUDA(nullptr, cudaMemcpyAsync(dst.scale, src.scale, p.sb, cudaMemcpyHostToDevice, h->s_in));
-            ECO_CUDA(nullptr, cudaMemcpyAsync(const_cast<void*>(dst.grad), src.grad, p.gb, cudaMemcpyHostToDevice, h->s_in));
-            ECO_CUDA(nullptr, cudaMemcpyAsync(dst.m, src.m, p.mb, cudaMemcpyHostToDevice, h->s_in));
-            up += p.wb + p.sb + p.gb + p.mb;
-            if (adam) { ECO_CUDA(nullptr, cudaMemcpyAsync(dst.v, src.v, p.mb, cudaMemcpyHostToDevice, h->s_in)); up += p.mb; }
+        for (const eco_host_ctx::Copy& cp : h->copies_in[c]) {
+            ECO_CUDA(nullptr, cudaMemcpyAsync(cp.dev, cp.host, cp.bytes, cudaMemcpyHostToDevice, h->s_in));
+            up += cp.bytes;
         }
         ECO_CUDA(nullptr, cudaEventRecord(h->ev_in[c], h->s_in));
         ECO_CUDA(nullptr, cudaStreamWaitEvent(h->s_run, h->ev_in[c], 0));
@@ -806,14 +869,9 @@ eco_status eco_host_step(eco_host_ctx* h, float lr, float beta1, float beta2, fl
         if (rc != ECO_OK) { g_thread_error = h->ctxs[c]->err; cudaDeviceSynchronize(); return rc; }
         ECO_CUDA(nullptr, cudaEventRecord(h->ev_run[c], h->s_run));
         ECO_CUDA(nullptr, cudaStreamWaitEvent(h->s_out, h->ev_run[c], 0));
-        for (size_t i = first; i < last; ++i) {
-            const eco_host_ctx::Place& p = h->place[i];
-            const eco_tensor &dst = h->host[i], &src = h->dev[i];
-            ECO_CUDA(nullptr, cudaMemcpyAsync(dst.w, src.w, p.wb, cudaMemcpyDeviceToHost, h->s_out));
-            ECO_CUDA(nullptr, cudaMemcpyAsync(dst.scale, src.scale, p.sb, cudaMemcpyDeviceToHost, h->s_out));
-            ECO_CUDA(nullptr, cudaMemcpyAsync(dst.m, src.m, p.mb, cudaMemcpyDeviceToHost, h->s_out));
-            down += p.wb + p.sb + p.mb;
-            if (adam) { ECO_CUDA(nullptr, cudaMemcpyAsync(dst.v, src.v, p.mb, cudaMemcpyDeviceToHost, h->s_out)); down += p.mb; }
+        for (const eco_host_ctx::Copy& cp : h->copies_out[c]) {
+            ECO_CUDA(nullptr, cudaMemcpyAsync(cp.host, cp.dev, cp.bytes, cudaMemcpyDeviceToHost, h->s_out));
+            down += cp.bytes;
         }
         ECO_CUDA(nullptr, cudaEventRecord(h->ev_out[c], h->s_out));
     }

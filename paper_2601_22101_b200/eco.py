@@ -24,7 +24,7 @@ ECO_OPT_SGDM, ECO_OPT_ADAM = 0, 1
 ECO_ROUND_NEAREST, ECO_ROUND_STOCHASTIC = 0, 1
 ECO_INJECT_NONE, ECO_INJECT_ECO, ECO_INJECT_EXACT = 0, 1, 2
 
-EXPORTED = ("eco_create", "eco_step", "eco_step_ex", "eco_step_begin", "eco_amax_buffer", "eco_step_end", "eco_step_host", "eco_host_create", "eco_host_step", "eco_host_destroy",
+EXPORTED = ("eco_create", "eco_step", "eco_step_ex", "eco_step_begin", "eco_amax_buffer", "eco_step_end", "eco_step_host", "eco_host_create", "eco_host_step", "eco_host_copies", "eco_host_destroy",
             "eco_step_static", "eco_check", "eco_attach_error_buffers", "eco_selftest_wait", "eco_destroy", "eco_last_error", "eco_quantize", "eco_dequantize",
             "eco_set_option", "eco_num_launches", "eco_version")
 
@@ -92,6 +92,8 @@ def load_library() -> ctypes.CDLL:
                                       ctypes.c_size_t, ctypes.c_int]
         L.eco_host_step.restype = ctypes.c_int
         L.eco_host_step.argtypes = [vp, f32, f32, f32, f32, u64, u64, ctypes.POINTER(u64), ctypes.POINTER(u64)]
+        L.eco_host_copies.restype = ctypes.c_int
+        L.eco_host_copies.argtypes = [vp, ctypes.POINTER(u64), ctypes.POINTER(u64)]
         L.eco_host_destroy.restype = ctypes.c_int
         L.eco_host_destroy.argtypes = [vp]
         L.eco_step_static.restype = ctypes.c_int
@@ -282,6 +284,15 @@ def eco_host_step(handle: int, lr: float, beta1: float, beta2: float, eps: float
     st = load_library().eco_host_step(handle, lr, beta1, beta2, eps, step, seed, ctypes.byref(up), ctypes.byref(down))
     if st != ECO_OK:
         _raise(st)
+    return up.value, down.value
+
+
+def eco_host_copies(handle: int):
+    """(h2d, d2h) copies one eco_host_step issues.  See include/eco.h."""
+    up, down = ctypes.c_uint64(0), ctypes.c_uint64(0)
+    st = load_library().eco_host_copies(handle, ctypes.byref(up), ctypes.byref(down))
+    if st != 0:
+        raise EcoError(st, "eco_host_copies")
     return up.value, down.value
 
 
