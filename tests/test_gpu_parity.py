@@ -437,21 +437,22 @@ def test_noise_floor_trends_of_sec_3_4_on_a_quadratic():
     assert floors["naive", 0.03] > 30 * floors["eco", 0.03]
 
 
-@pytest.mark.parametrize("fmt,opt", [(wl.FP8_E4M3, wl.ADAM), (wl.INT4, wl.SGDM)])
-def test_row_shards_with_amax_exchange_equal_the_unsplit_step(fmt, opt):
+@pytest.mark.parametrize("fmt,opt,sdt", [(wl.FP8_E4M3, wl.ADAM, wl.SCALE_F32), (wl.INT4, wl.SGDM, wl.SCALE_F32),
+                                         (wl.FP8_E5M2, wl.SGDM, wl.SCALE_E8M0)])
+def test_row_shards_with_amax_exchange_equal_the_unsplit_step(fmt, opt, sdt):
     """Per-tensor scales with tensors split by rows across ranks (emulated here as two contexts on one GPU, run
     one after the other: no kernel waits on another): pass 1 on each shard, element-wise maximum of the two amax
     vectors (what an all-reduce with MAX does), pass 2 on each shard.  With row_offset set the shards must hold
     exactly the bits of the unsplit step: same scale, same stochastic rounding per element."""
     shapes = [(64, 1024), (33, 384), (8, 640), (6, 200)]
-    w = _mini(fmt, wl.PER_TENSOR, wl.SCALE_F32, opt, wl.SR, shapes)
+    w = _mini(fmt, wl.PER_TENSOR, sdt, opt, wl.SR, shapes)
     full = DeviceState(w)
     full.init_from_host()
     full.create()
     adam = opt == wl.ADAM
     shards = []          # per rank: (tensors, handle)
     cuts = [t.rows // 2 for t in w.tensors]
-    per_row = lambda t: t.cols if fmt == wl.FP8_E4M3 else t.cols // 2
+    per_row = lambda t: t.cols // 2 if fmt == wl.INT4 else t.cols
     for rank in range(2):
         ts = []
         for i, (spec, d) in enumerate(zip(w.tensors, full.tensors)):
@@ -485,7 +486,7 @@ def test_row_shards_with_amax_exchange_equal_the_unsplit_step(fmt, opt):
             for i, (spec, d) in enumerate(zip(w.tensors, full.tensors)):
                 a, b = shards[0][0][i], shards[1][0][i]
                 assert torch.equal(torch.cat([a.w, b.w]), d.w), f"step {step} tensor {i}: codes"
-                assert torch.equal(a.scale.view(torch.int32), d.scale.view(torch.int32)) and torch.equal(a.scale, b.scale)
+                assert (_scale_bits(a.scale) == _scale_bits(d.scale)).all() and torch.equal(a.scale, b.scale)
                 assert torch.equal(torch.cat([a.m, b.m]), d.m), f"step {step} tensor {i}: m"
                 if adam:
                     assert torch.equal(torch.cat([a.v, b.v]), d.v)
@@ -506,14 +507,17 @@ def test_per_row_scales_on_long_and_short_rows(fmt, sdt, opt):
     run_chained(_mini(fmt, wl.PER_ROW, sdt, opt, wl.SR, shapes), steps=5)
 
 
-@pytest.mark.parametrize("fmt,gran,rnd", [(wl.FP8_E4M3, wl.PER_BLOCK, wl.SR), (wl.FP8_E4M3, wl.PER_TENSOR, wl.RTN),
-                                          (wl.INT4, wl.PER_ROW, wl.SR)])
+@pytest.mark.parametrize("fmt,gran,rnd,sdt,block", [(wl.FP8_E4M3, wl.PER_BLOCK, wl.SR, wl.SCALE_F32, 128),
+                                                    (wl.FP8_E4M3, wl.PER_TENSOR, wl.RTN, wl.SCALE_F32, 128),
+                                                    (wl.INT4, wl.PER_ROW, wl.SR, wl.SCALE_F32, 128),
+                                                    (wl.FP8_E4M3, wl.PER_BLOCK, wl.SR, wl.SCALE_E8M0, 32),
+                                                    (wl.FP8_E5M2, wl.PER_BLOCK, wl.RTN, wl.SCALE_BF16, 32)])
 @pytest.mark.parametrize("injection", [eco.ECO_INJECT_EXACT, eco.ECO_INJECT_ECO])
-def test_error_buffers_and_exact_injection(fmt, gran, rnd, injection):
+def test_error_buffers_and_exact_injection(fmt, gran, rnd, sdt, block, injection):
     """Attached error buffers receive e_{t+1} of every element at each step; ECO_INJECT_EXACT (Appendix A) reads them
     back as e_t.  Both against the oracle, which pins the exact rule to master-weight momentum SGD on the CPU."""
-    shapes = RAGGED + (RAGGED_FP8_ONLY if fmt == wl.FP8_E4M3 else [])
-    w = _mini(fmt, gran, wl.SCALE_F32, wl.SGDM, rnd, shapes)
+    shapes = RAGGED + (RAGGED_FP8_ONLY if fmt != wl.INT4 else [])
+    w = _mini(fmt, gran, sdt, wl.SGDM, rnd, shapes, block=block)
     dev = DeviceState(w)
     dev.init_from_host()
     ora = OracleState(w, injection=oracle.INJECT_IDEAL if injection == eco.ECO_INJECT_EXACT else oracle.INJECT_ECO)
