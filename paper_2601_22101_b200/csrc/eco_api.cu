@@ -211,6 +211,7 @@ StepParams derive_params(const eco_config& cfg, float lr_f, float beta1_f, float
     P.seed_hi = static_cast<uint32_t>(seed >> 32);
     P.step_lo = static_cast<uint32_t>(step);
     P.step_hi = static_cast<uint32_t>(step >> 32);
+    P.exact_qs = cfg.scale_dtype != ECO_SCALE_F32 ? 1 : 0;
     P.inject = cfg.injection == ECO_INJECT_ECO ? 1 : (cfg.injection == ECO_INJECT_EXACT ? 2 : 0);
     P.inv_lr = static_cast<float>(1.0 / lr);
     P.inv_lr_beta = static_cast<float>(1.0 / (lr * b1));

@@ -175,7 +175,10 @@ __device__ __forceinline__ bool consume_unit(const StepParams& P, const int scal
             float val[4];
             unpack4<FMT>(codes, val);
 #pragma unroll
-            for (int e = 0; e < 4; ++e) th[k][e] = __fmul_rn(val[e], s_old);
+            for (int p = 0; p < 4; p += 2) {
+                const float2 t = mul2(make_float2(val[p], val[p + 1]), dup2(s_old));
+                th[k][p] = t.x; th[k][p + 1] = t.y;
+            }
         }
         optim_rows<OPT, NS>(P, th, g, m, v, L, vt);
 #pragma unroll
