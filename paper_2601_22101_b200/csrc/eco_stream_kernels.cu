@@ -313,7 +313,10 @@ __device__ __forceinline__ bool consume_unit(const StepParams& P, const int scal
             const float4 er = *reinterpret_cast<const float4*>(ep + i0);
             e_prev[0] = er.x; e_prev[1] = er.y; e_prev[2] = er.z; e_prev[3] = er.w;
         }
-        const uint32_t codes = back4<FMT, OPT, RND, ERR>(P, word, s_k[k], inv_k[k], L[k], mh, e_prev, e_out);
+        // power-of-two scales make q s exact; INT4 kernels ask the step parameters (bf16 scales do too); the 8-bit
+        // float kernels with f32 / bf16 scales take the two-operation form without asking
+        constexpr int kExact = MODE == MODE_BLOCK32 ? 1 : (FMT == FMT_INT4 ? -1 : 0);
+        const uint32_t codes = back4<FMT, OPT, RND, ERR, kExact>(P, word, s_k[k], inv_k[k], L[k], mh, e_prev, e_out);
         if (FMT != FMT_INT4) *reinterpret_cast<uint32_t*>(wp + i0) = codes;
         else *reinterpret_cast<uint16_t*>(wp + (i0 >> 1)) = static_cast<uint16_t>(codes);
         *reinterpret_cast<float4*>(mp + i0) = make_float4(mh[0], mh[1], mh[2], mh[3]);
