@@ -683,3 +683,58 @@ def test_moments_match_bit_for_bit(fmt, sdt, opt, gran, monkeypatch):
     shapes = RAGGED + (RAGGED_FP8_ONLY if fmt != wl.INT4 else []) + [(40, 512)]
     run_chained(_mini(fmt, gran, sdt, opt, wl.SR, shapes), steps=8)
     run_chained(_mini(fmt, gran, sdt, opt, wl.RTN, shapes, lr=3e-3, grad_std=3e-2), steps=3, weight_decay=0.1, grad_scale=0.37)
+
+
+def test_tensor_with_more_than_2_to_the_32_elements():
+    """One tensor of 2^32 + 2^20 elements (INT4, group-128 bf16 scales, momentum SGD, stochastic rounding; 28 GB of
+    state): element offsets and the random-stream counters need more than 32 bits.  Checked on row slices: the first
+    rows against the oracle (their global indices are local ones), and rows on both sides of element 2^32 and the last
+    rows against a small context over a COPY of the slice with row_offset set, whose own arithmetic stays below 2^32
+    (that form is held to the oracle by test_row_shards_with_amax_exchange_equal_the_unsplit_step)."""
+    rows, cols = (1 << 22) + 1024, 1024
+    spec = wl.TensorSpec("huge", rows, cols, 7)
+    w = wl.Workload("huge_int4", wl.INT4, wl.PER_BLOCK, 128, wl.SCALE_BF16, wl.SGDM, wl.SR, lr=5e-2, beta1=0.9, beta2=0.95,
+                    eps=1e-8, weight_std=0.02, grad_std=5e-2, steps=1, step_seed=0x1234567, tensors=[spec])
+    free, _ = torch.cuda.mem_get_info()
+    if free < 60 * 2 ** 30:
+        pytest.skip("needs about 50 GB of device memory")
+    dev = DeviceState(w)
+    dev.init_on_device(seed=3)
+    dev.set_grads_on_device(seed=4)
+    d = dev.tensors[0]
+    d.m.normal_(0.0, 1e-4)
+    boundary = (1 << 32) // cols
+    slices = [(0, 8), (boundary - 4, boundary + 4), (rows - 8, rows)]
+    before = []
+    for r0, r1 in slices:
+        e0, e1 = r0 * cols, r1 * cols
+        before.append((d.w[e0 // 2: e1 // 2].clone(), d.scale[r0 * 8: r1 * 8].clone(), d.grad[e0: e1].clone(), d.m[e0: e1].clone()))
+    dev.create()
+    try:
+        dev.step(1)
+        torch.cuda.synchronize()
+        eco.eco_check(dev.handle, torch.cuda.current_stream().cuda_stream)
+        for (r0, r1), (bw, bs, bg, bm) in zip(slices, before):
+            e0, e1 = r0 * cols, r1 * cols
+            shard = eco.Tensor(bw.clone(), bs.clone(), bg, bm.clone(), None, r1 - r0, cols, spec.tensor_id, row_offset=r0)
+            h = eco.eco_create(config_of(w), [shard])
+            try:
+                eco.eco_step(h, w.lr, w.beta1, w.beta2, w.eps, 1, w.step_seed, torch.cuda.current_stream().cuda_stream)
+                torch.cuda.synchronize()
+            finally:
+                eco.eco_destroy(h)
+            assert torch.equal(shard.w, d.w[e0 // 2: e1 // 2]), f"rows {r0}..{r1}: codes"
+            assert torch.equal(shard.scale.view(torch.int16), d.scale[r0 * 8: r1 * 8].view(torch.int16)), f"rows {r0}..{r1}: scales"
+            assert torch.equal(shard.m, d.m[e0: e1]), f"rows {r0}..{r1}: m"
+            assert not torch.equal(shard.w, bw)                                        # the step did change the codes
+        # first rows against the oracle
+        bw, bs, bg, bm = before[0]
+        cw, cs = _np(bw).copy(), _np(bs.view(torch.int16)).view(np.uint16).copy()
+        cg, cm = _np(bg.view(torch.int16)).view(np.uint16).copy(), _np(bm).copy()
+        oracle.step(oracle_config(w), lr=float(np.float32(w.lr)), beta1=float(np.float32(w.beta1)), beta2=float(np.float32(w.beta2)),
+                    eps=float(np.float32(w.eps)), step=1, seed=w.step_seed, w=cw, scale=cs, grad=cg, m=cm, v=None,
+                    rows=8, cols=cols, tensor_id=spec.tensor_id)
+        assert (_np(d.w[: 8 * cols // 2]) == cw).all() and (_np(d.scale[: 64].view(torch.int16)).view(np.uint16) == cs).all()
+        assert (_np(d.m[: 8 * cols]).view(np.int32) == cm.view(np.int32)).all()
+    finally:
+        dev.destroy()
