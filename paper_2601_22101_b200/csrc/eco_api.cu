@@ -257,6 +257,8 @@ eco_status eco_create(eco_ctx** out, const eco_config* cfg, const eco_tensor* te
     if (eco_status st = check_config(cfg, true)) return st;
     if (!tensors || n == 0) return fail(nullptr, ECO_ERR_INVALID_ARG, "empty tensor list");
     if (n > 0x7FFFFFFFu) return fail(nullptr, ECO_ERR_INVALID_ARG, "too many tensors");
+    for (size_t i = 0; i < n; ++i)                       // what needs no device is refused before any CUDA call
+        if (eco_status st = check_shape(*cfg, tensors[i].rows, tensors[i].cols, i)) return st;
     ECO_CUDA(nullptr, cudaSetDevice(device));
     cudaDeviceProp prop;
     ECO_CUDA(nullptr, cudaGetDeviceProperties(&prop, device));

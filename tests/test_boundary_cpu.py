@@ -50,7 +50,22 @@ def test_validation_rejects_before_touching_cuda(lib):
         eco.eco_create(eco.Config(block=64), [eco.Tensor(None, None, None, None, None, 1, 1, 0)])
     assert e.value.status == eco.ECO_ERR_UNSUPPORTED and "128" in str(e.value)
     with pytest.raises(eco.EcoError) as e:
+        eco.eco_create(eco.Config(scale_dtype=3), [eco.Tensor(None, None, None, None, None, 1, 1, 0)])
+    assert e.value.status == eco.ECO_ERR_UNSUPPORTED
+    with pytest.raises(eco.EcoError) as e:
         eco.eco_create(eco.Config(), [])
+    assert e.value.status == eco.ECO_ERR_INVALID_ARG
+    # the configurations added beside the paper's own (E5M2, 1x32 blocks, power-of-two scales) pass the configuration
+    # check: what is refused next is the empty tensor (rows = 0), an argument error
+    for cfg in (eco.Config(format=eco.ECO_FORMAT_FP8_E5M2), eco.Config(block=32, scale_dtype=eco.ECO_SCALE_E8M0)):
+        with pytest.raises(eco.EcoError) as e:
+            eco.eco_create(cfg, [eco.Tensor(None, None, None, None, None, 0, 128, 0)])
+        assert e.value.status == eco.ECO_ERR_INVALID_ARG and "rows" in str(e.value)
+    with pytest.raises(eco.EcoError) as e:                    # more than 2^34 elements
+        eco.eco_create(eco.Config(), [eco.Tensor(None, None, None, None, None, 1 << 20, 1 << 14, 0)])
+    assert e.value.status == eco.ECO_ERR_INVALID_ARG and "2^34" in str(e.value)
+    with pytest.raises(eco.EcoError) as e:                    # INT4 packs two codes per byte
+        eco.eco_create(eco.Config(format=eco.ECO_FORMAT_INT4), [eco.Tensor(None, None, None, None, None, 4, 127, 0)])
     assert e.value.status == eco.ECO_ERR_INVALID_ARG
     with pytest.raises(eco.EcoError) as e:
         eco.eco_step(None, 1e-3, 0.9, 0.95, 1e-8, 1, 0)
