@@ -17,6 +17,8 @@
 //                        order-free); pass 2 recomputes theta~ and finishes.
 //   per-row scale      : one CTA per row, two loops over the row (the second
 //                        loop re-reads the row from L1/L2).
+#include <algorithm>
+
 #include "eco_device.cuh"
 #include "eco_launch.h"
 
@@ -488,8 +490,77 @@ eco_dequantize_kernel(const uint8_t* __restrict__ w, const void* __restrict__ sc
     }
 }
 
+// The same for rows whose length is a multiple of 16 and 16-byte aligned buffers: one thread per EPT consecutive
+// elements (they share a scale: 4, 8 and 16 divide both block lengths).  EPT is chosen so that a lane stores exactly
+// 16 bytes, contiguous with its neighbours': 8 elements for bf16 output, 4 for f32.
+template <int FMT, bool OUT_BF16, int EPT>
+__global__ void __launch_bounds__(kThreads)
+eco_dequantize_vec_kernel(const uint8_t* __restrict__ w, const void* __restrict__ scale, void* __restrict__ out,
+                          const uint32_t n_units, const uint32_t units_per_row, const int gran, const uint32_t block,
+                          const uint32_t scales_per_row, const int scale_kind) {
+    static_assert(EPT == 4 || EPT == 8, "4 or 8 elements per thread");
+    constexpr int Q = EPT / 4;
+    for (uint32_t u = blockIdx.x * kThreads + threadIdx.x; u < n_units; u += gridDim.x * kThreads) {
+        const uint32_t row = u / units_per_row, c0 = (u - row * units_per_row) * EPT;
+        const uint64_t i0 = static_cast<uint64_t>(u) * EPT;
+        uint32_t codes[Q];
+        if (FMT != FMT_INT4) {
+            if constexpr (EPT == 8) {
+                const uint2 r = __ldg(reinterpret_cast<const uint2*>(w + i0));
+                codes[0] = r.x; codes[1] = r.y;
+            } else {
+                codes[0] = __ldg(reinterpret_cast<const uint32_t*>(w + i0));
+            }
+        } else {
+            if constexpr (EPT == 8) {
+                const uint32_t r = __ldg(reinterpret_cast<const uint32_t*>(w + (i0 >> 1)));
+                codes[0] = r & 0xFFFFu; codes[1] = r >> 16;
+            } else {
+                codes[0] = __ldg(reinterpret_cast<const uint16_t*>(w + (i0 >> 1)));
+            }
+        }
+        const uint64_t k = gran == 0 ? 0 : (gran == 1 ? row : static_cast<uint64_t>(row) * scales_per_row + c0 / block);
+        const float s = load_scale(scale, k, scale_kind);
+        float x[EPT];
+#pragma unroll
+        for (int q = 0; q < Q; ++q) {
+            float val[4];
+            unpack4<FMT>(codes[q], val);
+#pragma unroll
+            for (int e = 0; e < 4; ++e) x[4 * q + e] = __fmul_rn(val[e], s);
+        }
+        if (OUT_BF16) {
+            uint32_t p[EPT / 2];
+#pragma unroll
+            for (int j = 0; j < EPT / 2; ++j)
+                p[j] = f32_to_bf16_bits_rne(x[2 * j]) | (f32_to_bf16_bits_rne(x[2 * j + 1]) << 16);
+            uint4* o = reinterpret_cast<uint4*>(static_cast<uint16_t*>(out) + i0);
+#pragma unroll
+            for (int j = 0; j < (EPT + 7) / 8; ++j) o[j] = make_uint4(p[4 * j], p[4 * j + 1], p[4 * j + 2], p[4 * j + 3]);
+        } else {
+            float4* o = reinterpret_cast<float4*>(static_cast<float*>(out) + i0);
+#pragma unroll
+            for (int j = 0; j < Q; ++j) o[j] = make_float4(x[4 * j], x[4 * j + 1], x[4 * j + 2], x[4 * j + 3]);
+        }
+    }
+}
+
 cudaError_t launch_dequantize(const LaunchConfig& c, const uint8_t* w, const void* scale, void* out, uint64_t rows,
                               uint32_t cols, int gran, bool out_bf16, uint32_t grid, cudaStream_t stream) {
+    const uint32_t block = static_cast<uint32_t>(128 / c.sub);
+    const bool aligned = ((reinterpret_cast<uintptr_t>(w) | reinterpret_cast<uintptr_t>(out)) & 15u) == 0;
+    if (cols % 16 == 0 && aligned) {
+        const uint32_t ept = out_bf16 ? 8u : 4u;                       // rows * cols < 2^34: unit indices fit 32 bits
+        const uint32_t n_units = static_cast<uint32_t>(rows * cols / ept);
+        const uint32_t cap = static_cast<uint32_t>((c.sm_count > 0 ? c.sm_count : 148) * 16);
+        const uint32_t g = std::max(1u, std::min(cap, (n_units + kThreads - 1) / kThreads));
+        const uint32_t spr = (cols + block - 1) / block;
+        ECO_DISPATCH_FMT(c.format, {
+            if (out_bf16) eco_dequantize_vec_kernel<F, true, 8><<<g, kThreads, 0, stream>>>(w, scale, out, n_units, cols / 8, gran, block, spr, c.scale_kind);
+            else eco_dequantize_vec_kernel<F, false, 4><<<g, kThreads, 0, stream>>>(w, scale, out, n_units, cols / 4, gran, block, spr, c.scale_kind);
+        })
+        return cudaGetLastError();
+    }
     ECO_DISPATCH_FMT(c.format, {
         if (out_bf16) eco_dequantize_kernel<F, true><<<grid, kThreads, 0, stream>>>(w, scale, out, rows, cols, gran, static_cast<uint32_t>(128 / c.sub), c.scale_kind);
         else eco_dequantize_kernel<F, false><<<grid, kThreads, 0, stream>>>(w, scale, out, rows, cols, gran, static_cast<uint32_t>(128 / c.sub), c.scale_kind);
