@@ -8,6 +8,7 @@ it with g++ and marshals numpy arrays.
 """
 from __future__ import annotations
 
+import contextlib
 import ctypes
 import os
 import subprocess
@@ -73,28 +74,46 @@ class Config:
 _lib = None
 
 
+def _bind(path: str) -> ctypes.CDLL:
+    L = ctypes.CDLL(path)
+    L.eco_oracle_element_random_word.restype = ctypes.c_uint32
+    L.eco_oracle_element_random_word.argtypes = [ctypes.c_uint64, ctypes.c_uint64, ctypes.c_uint32, ctypes.c_uint64]
+    L.eco_oracle_code_value.restype = ctypes.c_double
+    L.eco_oracle_code_value.argtypes = [ctypes.c_int, ctypes.c_int]
+    L.eco_oracle_f32_to_bf16.restype = ctypes.c_uint16
+    L.eco_oracle_f32_to_bf16.argtypes = [ctypes.c_float]
+    vp, u64, u32, dbl = ctypes.c_void_p, ctypes.c_uint64, ctypes.c_uint32, ctypes.c_double
+    L.eco_oracle_philox4x32_10.argtypes = [vp, vp, vp]
+    for sfx in ("f32", "f64"):
+        getattr(L, f"eco_oracle_round_{sfx}").argtypes = [ctypes.c_int, ctypes.c_int, vp, vp, u64, vp]
+        getattr(L, f"eco_oracle_quantize_{sfx}").argtypes = [vp, vp, u64, u64, vp, vp, u64, u64, u32, u64]
+        getattr(L, f"eco_oracle_dequantize_{sfx}").argtypes = [vp, vp, vp, u64, u64, vp]
+        getattr(L, f"eco_oracle_step_{sfx}").argtypes = [
+            vp, dbl, dbl, dbl, dbl, u64, u64, vp, vp, vp, vp, vp, u64, u64, u32, vp, vp, vp, vp, u64]
+        getattr(L, f"eco_oracle_step_ex_{sfx}").argtypes = [
+            vp, dbl, dbl, dbl, dbl, dbl, dbl, u64, u64, vp, vp, vp, vp, vp, u64, u64, u32, u64]
+    return L
+
+
 def lib() -> ctypes.CDLL:
     global _lib
     if _lib is None:
-        L = ctypes.CDLL(build())
-        L.eco_oracle_element_random_word.restype = ctypes.c_uint32
-        L.eco_oracle_element_random_word.argtypes = [ctypes.c_uint64, ctypes.c_uint64, ctypes.c_uint32, ctypes.c_uint64]
-        L.eco_oracle_code_value.restype = ctypes.c_double
-        L.eco_oracle_code_value.argtypes = [ctypes.c_int, ctypes.c_int]
-        L.eco_oracle_f32_to_bf16.restype = ctypes.c_uint16
-        L.eco_oracle_f32_to_bf16.argtypes = [ctypes.c_float]
-        vp, u64, u32, dbl = ctypes.c_void_p, ctypes.c_uint64, ctypes.c_uint32, ctypes.c_double
-        L.eco_oracle_philox4x32_10.argtypes = [vp, vp, vp]
-        for sfx in ("f32", "f64"):
-            getattr(L, f"eco_oracle_round_{sfx}").argtypes = [ctypes.c_int, ctypes.c_int, vp, vp, u64, vp]
-            getattr(L, f"eco_oracle_quantize_{sfx}").argtypes = [vp, vp, u64, u64, vp, vp, u64, u64, u32]
-            getattr(L, f"eco_oracle_dequantize_{sfx}").argtypes = [vp, vp, vp, u64, u64, vp]
-            getattr(L, f"eco_oracle_step_{sfx}").argtypes = [
-                vp, dbl, dbl, dbl, dbl, u64, u64, vp, vp, vp, vp, vp, u64, u64, u32, vp, vp, vp, vp]
-            getattr(L, f"eco_oracle_step_ex_{sfx}").argtypes = [
-                vp, dbl, dbl, dbl, dbl, dbl, dbl, u64, u64, vp, vp, vp, vp, vp, u64, u64, u32]
-        _lib = L
+        _lib = _bind(build())
     return _lib
+
+
+@contextlib.contextmanager
+def use_library(path: str):
+    """Route every call of this module to another build of the oracle for the length of the block.  The
+    mutation tests use it: they compile a copy of eco_oracle.cpp with one mistake planted in it and check
+    that the pins notice."""
+    global _lib
+    saved = lib()
+    _lib = _bind(path)
+    try:
+        yield
+    finally:
+        _lib = saved
 
 
 def _ptr(a):
@@ -143,15 +162,16 @@ def scale_numpy_dtype(cfg: Config, real=np.float32):
     return {SCALE_BF16: np.uint16, SCALE_E8M0: np.uint8}.get(cfg.scale_dtype, real)
 
 
-def quantize(cfg: Config, x: np.ndarray, seed: int = 0, step: int = 0, tensor_id: int = 0):
-    """theta_hat = q(x) for a [rows, cols] array; returns (codes, scales)."""
+def quantize(cfg: Config, x: np.ndarray, seed: int = 0, step: int = 0, tensor_id: int = 0, index_base: int = 0):
+    """theta_hat = q(x) for a [rows, cols] array; returns (codes, scales).  ``index_base``: position of
+    x[0, 0] inside the full tensor when x is a slice of whole rows of it (random words are drawn per position)."""
     x = np.ascontiguousarray(x)
     rows, cols = x.shape
     w = np.zeros(cfg.code_bytes(rows, cols), dtype=np.uint8)
     s = np.zeros(cfg.n_scales(rows, cols), dtype=scale_numpy_dtype(cfg, x.dtype))
     c = cfg.c()
     rc = getattr(lib(), f"eco_oracle_quantize_{_sfx(x.dtype)}")(
-        ctypes.byref(c), _ptr(x), rows, cols, _ptr(w), _ptr(s), seed, step, tensor_id)
+        ctypes.byref(c), _ptr(x), rows, cols, _ptr(w), _ptr(s), seed, step, tensor_id, index_base)
     assert rc == 0
     return w, s
 
@@ -169,20 +189,21 @@ def step(cfg: Config, *, lr: float, beta1: float, beta2: float = 0.0, eps: float
          m: np.ndarray, v: np.ndarray | None = None, rows: int, cols: int, tensor_id: int = 0,
          noise: np.ndarray | None = None, e_prev: np.ndarray | None = None,
          dbg_theta_tilde: np.ndarray | None = None, dbg_err: np.ndarray | None = None,
-         weight_decay: float = 0.0, grad_scale: float = 1.0) -> None:
+         weight_decay: float = 0.0, grad_scale: float = 1.0, index_base: int = 0) -> None:
     """One Algorithm-1 step on one tensor, in place.  ``m.dtype`` selects binary32 or binary64.
     ``weight_decay`` (decoupled, AdamW style) and ``grad_scale`` (one factor on the gradient, e.g. the
-    clipping factor) are the two additions of Sec. 4's training recipe to OPTIM_STEP."""
+    clipping factor) are the two additions of Sec. 4's training recipe to OPTIM_STEP.  ``index_base``: position of
+    the buffers' first element inside the full tensor when they hold a slice of whole rows of it."""
     c = cfg.c()
     if weight_decay != 0.0 or grad_scale != 1.0:
         assert noise is None and e_prev is None and dbg_theta_tilde is None and dbg_err is None
         rc = getattr(lib(), f"eco_oracle_step_ex_{_sfx(m.dtype)}")(
             ctypes.byref(c), float(lr), float(beta1), float(beta2), float(eps), float(weight_decay), float(grad_scale),
-            int(step), int(seed), _ptr(w), _ptr(scale), _ptr(grad), _ptr(m), _ptr(v), rows, cols, tensor_id)
+            int(step), int(seed), _ptr(w), _ptr(scale), _ptr(grad), _ptr(m), _ptr(v), rows, cols, tensor_id, int(index_base))
         assert rc == 0
         return
     rc = getattr(lib(), f"eco_oracle_step_{_sfx(m.dtype)}")(
         ctypes.byref(c), float(lr), float(beta1), float(beta2), float(eps), int(step), int(seed),
         _ptr(w), _ptr(scale), _ptr(grad), _ptr(m), _ptr(v), rows, cols, tensor_id,
-        _ptr(noise), _ptr(e_prev), _ptr(dbg_theta_tilde), _ptr(dbg_err))
+        _ptr(noise), _ptr(e_prev), _ptr(dbg_theta_tilde), _ptr(dbg_err), int(index_base))
     assert rc == 0

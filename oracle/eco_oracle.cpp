@@ -22,9 +22,16 @@
 // by Monte Carlo; Philox against a library generator; identity quantizer ->
 // plain SGDM / Adam; Lemma 3.5 telescoping; the Adam one-step identity;
 // Appendix A exact equivalence with master weights; Appendix C stationary
-// second moments; power-of-two block scales against exact rational search,
-// a library decode of the exponent byte and power-of-two invariance.  The order of the binary32 operations is this build's
-// choice (the paper fixes none): parity unpinned for that order alone.
+// second moments of all three regimes (ECO, naive, master weights); the scale
+// s = max|x| / rho by its consequences (the largest element of every block
+// lands on +-rho, s * rho gives the maximum back) with block extents and code
+// layout written out independently; power-of-two block scales against exact
+// rational search, a library decode of the exponent byte and power-of-two
+// invariance; the position of a row slice in the random stream against the
+// whole tensor.  tests/test_oracle_mutations.py plants mistakes in a scratch
+// copy of this file and checks that those pins fail.  The order of the
+// binary32 operations is this build's choice (the paper fixes none): parity
+// unpinned for that order alone.
 
 #include <cmath>
 #include <cstdint>
@@ -315,10 +322,14 @@ void block_extent(const OracleConfig& cfg, const BlockGrid& g, uint64_t rows, ui
 // q(x): the symmetric quantizer of Sec. 3.1 applied block by block.  Used for
 // the initial state theta_hat_0 = q(theta_0) (Appendix A, initialisation) and
 // by the master-weight reference of the tests.
+// index_base: position of x[0] inside the full tensor when x is a slice of whole rows of it (0 for a
+// whole tensor); the random word of element i is the one of position index_base + i, so a slice
+// rounds exactly like the same rows inside the whole tensor.
 // ---------------------------------------------------------------------------
 template <class R>
 int quantize_tensor(const OracleConfig& cfg, const R* x, uint64_t rows, uint64_t cols,
-                    uint8_t* w, void* scale, uint64_t seed, uint64_t step, uint32_t tensor_id) {
+                    uint8_t* w, void* scale, uint64_t seed, uint64_t step, uint32_t tensor_id,
+                    uint64_t index_base) {
     const BlockGrid g = block_grid(cfg, rows, cols);
     for (uint64_t k = 0; k < g.n_blocks; ++k) {
         uint64_t begin, len;
@@ -331,7 +342,7 @@ int quantize_tensor(const OracleConfig& cfg, const R* x, uint64_t rows, uint64_t
         R s, inv;
         make_scale<R>(cfg.format, cfg.scale_dtype, amax, scale, k, &s, &inv);
         for (uint64_t i = begin; i < begin + len; ++i) {
-            const uint32_t r = cfg.rounding == ROUND_SR ? element_random_word(seed, step, tensor_id, i) : 0u;
+            const uint32_t r = cfg.rounding == ROUND_SR ? element_random_word(seed, step, tensor_id, index_base + i) : 0u;
             store_code(cfg.format, w, i, round_to_code<R>(cfg.format, cfg.rounding, x[i] * inv, r));
         }
     }
@@ -366,6 +377,9 @@ struct Hyper {
     // factor min(1, c / ||g||), computed by the caller).  0 and 1 switch them off.
     double weight_decay = 0.0;
     double grad_scale = 1.0;
+    // Position of the buffers' first element inside the full tensor when they hold a slice of whole rows of it
+    // (0 for a whole tensor): element i draws the random word of position index_base + i.
+    uint64_t index_base = 0;
 };
 
 template <class R>
@@ -479,7 +493,7 @@ int step_tensor(const OracleConfig& cfg, const Hyper& hyper,
             R thq;
             if (coded) {
                 const uint32_t r = cfg.rounding == ROUND_SR
-                                       ? element_random_word(hyper.seed, hyper.step, tensor_id, i) : 0u;
+                                       ? element_random_word(hyper.seed, hyper.step, tensor_id, hyper.index_base + i) : 0u;
                 const int code = round_to_code<R>(cfg.format, cfg.rounding, tht * inv, r);
                 store_code(cfg.format, static_cast<uint8_t*>(w), i, code);
                 thq = code_value<R>(cfg.format, code) * s;
@@ -536,12 +550,14 @@ void eco_oracle_round_f64(int format, int rounding, const double* y, const uint3
 uint16_t eco_oracle_f32_to_bf16(float f) { return f32_to_bf16_rne(f); }
 
 int eco_oracle_quantize_f32(const OracleConfig* cfg, const float* x, uint64_t rows, uint64_t cols,
-                            uint8_t* w, void* scale, uint64_t seed, uint64_t step, uint32_t tensor_id) {
-    return quantize_tensor<float>(*cfg, x, rows, cols, w, scale, seed, step, tensor_id);
+                            uint8_t* w, void* scale, uint64_t seed, uint64_t step, uint32_t tensor_id,
+                            uint64_t index_base) {
+    return quantize_tensor<float>(*cfg, x, rows, cols, w, scale, seed, step, tensor_id, index_base);
 }
 int eco_oracle_quantize_f64(const OracleConfig* cfg, const double* x, uint64_t rows, uint64_t cols,
-                            uint8_t* w, void* scale, uint64_t seed, uint64_t step, uint32_t tensor_id) {
-    return quantize_tensor<double>(*cfg, x, rows, cols, w, scale, seed, step, tensor_id);
+                            uint8_t* w, void* scale, uint64_t seed, uint64_t step, uint32_t tensor_id,
+                            uint64_t index_base) {
+    return quantize_tensor<double>(*cfg, x, rows, cols, w, scale, seed, step, tensor_id, index_base);
 }
 int eco_oracle_dequantize_f32(const OracleConfig* cfg, const uint8_t* w, const void* scale,
                               uint64_t rows, uint64_t cols, float* x) {
@@ -556,16 +572,18 @@ int eco_oracle_step_f32(const OracleConfig* cfg, double lr, double beta1, double
                         uint64_t step, uint64_t seed,
                         void* w, void* scale, const void* grad, float* m, float* v,
                         uint64_t rows, uint64_t cols, uint32_t tensor_id,
-                        const float* noise, float* e_prev, float* dbg_theta_tilde, float* dbg_err) {
-    const Hyper h{lr, beta1, beta2, eps, step, seed};
+                        const float* noise, float* e_prev, float* dbg_theta_tilde, float* dbg_err, uint64_t index_base) {
+    Hyper h{lr, beta1, beta2, eps, step, seed};
+    h.index_base = index_base;
     return step_tensor<float>(*cfg, h, w, scale, grad, m, v, rows, cols, tensor_id,
                               noise, e_prev, dbg_theta_tilde, dbg_err);
 }
 int eco_oracle_step_ex_f32(const OracleConfig* cfg, double lr, double beta1, double beta2, double eps,
                            double weight_decay, double grad_scale, uint64_t step, uint64_t seed,
                            void* w, void* scale, const void* grad, float* m, float* v,
-                           uint64_t rows, uint64_t cols, uint32_t tensor_id) {
+                           uint64_t rows, uint64_t cols, uint32_t tensor_id, uint64_t index_base) {
     Hyper h{lr, beta1, beta2, eps, step, seed};
+    h.index_base = index_base;
     h.weight_decay = weight_decay;
     h.grad_scale = grad_scale;
     return step_tensor<float>(*cfg, h, w, scale, grad, m, v, rows, cols, tensor_id, nullptr, nullptr, nullptr, nullptr);
@@ -573,8 +591,9 @@ int eco_oracle_step_ex_f32(const OracleConfig* cfg, double lr, double beta1, dou
 int eco_oracle_step_ex_f64(const OracleConfig* cfg, double lr, double beta1, double beta2, double eps,
                            double weight_decay, double grad_scale, uint64_t step, uint64_t seed,
                            void* w, void* scale, const void* grad, double* m, double* v,
-                           uint64_t rows, uint64_t cols, uint32_t tensor_id) {
+                           uint64_t rows, uint64_t cols, uint32_t tensor_id, uint64_t index_base) {
     Hyper h{lr, beta1, beta2, eps, step, seed};
+    h.index_base = index_base;
     h.weight_decay = weight_decay;
     h.grad_scale = grad_scale;
     return step_tensor<double>(*cfg, h, w, scale, grad, m, v, rows, cols, tensor_id, nullptr, nullptr, nullptr, nullptr);
@@ -583,8 +602,9 @@ int eco_oracle_step_f64(const OracleConfig* cfg, double lr, double beta1, double
                         uint64_t step, uint64_t seed,
                         void* w, void* scale, const void* grad, double* m, double* v,
                         uint64_t rows, uint64_t cols, uint32_t tensor_id,
-                        const double* noise, double* e_prev, double* dbg_theta_tilde, double* dbg_err) {
-    const Hyper h{lr, beta1, beta2, eps, step, seed};
+                        const double* noise, double* e_prev, double* dbg_theta_tilde, double* dbg_err, uint64_t index_base) {
+    Hyper h{lr, beta1, beta2, eps, step, seed};
+    h.index_base = index_base;
     return step_tensor<double>(*cfg, h, w, scale, grad, m, v, rows, cols, tensor_id,
                                noise, e_prev, dbg_theta_tilde, dbg_err);
 }

@@ -261,6 +261,50 @@ def test_appendix_c_stationary_second_moments():
     assert abs(eco_small / (sigma ** 2 / (1 - beta ** 2)) - 1) < 0.05
 
 
+def pin_master_weight_second_moments(chains=200000, steps=600, seed=17):
+    """Appendix C, master-weight regime: full-precision x is kept, the gradient is taken at x^ = x + xi, and the
+    update is plain SGDM on x (the oracle's step with the identity quantizer).  Stationary second moments against
+    the closed forms u, v, w of that subsection and E[x^^2] = u + sigma^2."""
+    gold = _golden("appendix_c_setting.txt")
+    L, lr, beta, sigma = gold["L"], gold["eta"], gold["beta"], gold["sigma"]
+    D = 2 * (1 + beta) - L * lr * (1 - beta)
+    u = L * lr * sigma ** 2 * (1 + beta) / D
+    v = L ** 2 * lr * sigma ** 2 * (beta - 1) / D
+    w = 2 * L ** 2 * sigma ** 2 * (1 - beta) / D
+    assert abs(u - gold["mw_u_expected"]) < 1e-6 and abs(v - gold["mw_v_expected"]) < 1e-6
+    assert abs(w - gold["mw_w_expected"]) < 1e-6 and abs(u + sigma ** 2 - gold["mw_xhat2_expected"]) < 1e-6
+    rng = np.random.default_rng(seed)
+    cfg = oracle.Config(format=IDENTITY, optimizer=SGDM, grad_dtype=GRAD_NATIVE)
+    x, m = np.zeros(chains), np.zeros(chains)
+    acc = np.zeros(4)
+    cnt = 0
+    for t in range(1, steps + 1):
+        xhat = x + rng.standard_normal(chains) * sigma
+        oracle.step(cfg, lr=lr, beta1=beta, step=t, w=x, scale=None, grad=L * xhat, m=m, rows=1, cols=chains)
+        if t > steps // 2:
+            nxt = x + rng.standard_normal(chains) * sigma            # what the model would see now (not fed back)
+            acc += [np.mean(x * x), np.mean(x * m), np.mean(m * m), np.mean(nxt * nxt)]
+            cnt += 1
+    gu, gv, gw, gx = acc / cnt
+    assert abs(gu / u - 1) < 0.02, (gu, u)
+    assert abs(gv / v - 1) < 0.05, (gv, v)
+    assert abs(gw / w - 1) < 0.02, (gw, w)
+    assert abs(gx / (u + sigma ** 2) - 1) < 0.01, (gx, u + sigma ** 2)
+
+
+def test_appendix_c_master_weight_regime():
+    pin_master_weight_second_moments()
+
+
+def test_appendix_c_orders_the_three_regimes():
+    """Sec. 3.4 at the golden setting: master weights sit at the quantization floor, ECO a constant factor above
+    it, naive removal higher still -- as closed forms and as the ratios the paper draws from them."""
+    gold = _golden("appendix_c_setting.txt")
+    assert gold["mw_xhat2_expected"] < gold["eco_expected"] < gold["naive_expected"]
+    beta, sigma = gold["beta"], gold["sigma"]
+    assert abs(gold["eco_expected"] / (sigma ** 2 / (1 - beta ** 2)) - 1) < 0.01     # eta -> 0 limit already close
+
+
 def test_memory_layout_matches_paper_count():
     """Sec. 4.4 (Discussion on Memory): 12 bytes per parameter with FP32 master weights, 9 without."""
     gold = _golden("paper_constants.txt")
