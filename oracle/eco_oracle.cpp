@@ -192,7 +192,8 @@ void lower_neighbour(int format, R a, int* lo_code, R* frac) {
 }
 
 // Round a scaled value y = x / s to a code of the format (Sec. 3.1, rounding
-// paragraph).  Magnitudes beyond rho are clamped to rho first; a NaN takes rho.
+// paragraph).  Magnitudes beyond rho are clamped to rho first; a NaN takes +rho
+// whatever its sign bit (IEEE 754 leaves the sign of a computed NaN open, and processors differ).
 //   RTN: the closest grid point, ties to the even code.
 //   SR : the upper neighbour with probability frac (the distance to the lower
 //        one over the gap), decided by comparing the top 24 bits of the
@@ -200,7 +201,7 @@ void lower_neighbour(int format, R a, int* lo_code, R* frac) {
 template <class R>
 int round_to_code(int format, int rounding, R y, uint32_t random_word) {
     const R rho = format_rho<R>(format);
-    const bool negative = std::signbit(y);
+    const bool negative = std::signbit(y) && !std::isnan(y);   // the sign bit of a NaN means nothing: it takes +rho
     const R ay = std::fabs(y);
     const R a = (ay < rho) ? ay : rho;
     int lo;

@@ -69,6 +69,11 @@ def test_saturation_and_never_nan_or_minus_eight():
         codes = oracle.round_to_codes(FP8_E4M3, mode, y, np.full(y.size, 1, np.uint32))
         assert all((c & 0x7F) == 0x7E for c in codes)
         assert list(codes[6:] >> 7) == [1, 1, 1]
+    # a NaN takes +rho whatever its sign bit (processors differ in the sign of the NaN an operation returns)
+    nans = np.array([0x7FC00000, 0xFFC00000, 0x7F800001, 0xFFFFFFFF], np.uint32).view(np.float32)
+    for mode in (RTN, SR):
+        assert list(oracle.round_to_codes(FP8_E4M3, mode, nans, np.zeros(4, np.uint32))) == [0x7E] * 4
+        assert list(oracle.round_to_codes(INT4, mode, nans, np.zeros(4, np.uint32))) == [7] * 4
     y4 = np.array([7.0, 7.4, 7.5, 8.0, 100.0, np.inf, -7.5, -100.0], dtype=np.float32)
     for mode in (RTN, SR):
         codes = oracle.round_to_codes(INT4, mode, y4, np.zeros(y4.size, np.uint32))
