@@ -107,8 +107,8 @@ typedef struct eco_tensor {
  *   device   CUDA device ordinal; made current for the calling thread.
  * Errors: ECO_ERR_INVALID_ARG (NULL, n == 0, rows/cols < 1, rows*cols >= 2^34,
  * INT4 with odd cols, duplicate tensor_id, v not matching the optimizer,
- * overlapping buffers, non-device pointers), ECO_ERR_UNSUPPORTED (block != 128,
- * unknown enum), ECO_ERR_ALIGNMENT, ECO_ERR_CUDA, ECO_ERR_NOMEM.  On error *out
+ * overlapping buffers, non-device pointers), ECO_ERR_UNSUPPORTED (a block other
+ * than 128 or 32, unknown enum), ECO_ERR_ALIGNMENT, ECO_ERR_CUDA, ECO_ERR_NOMEM.  On error *out
  * is NULL and eco_last_error(NULL) describes the failure.  Allocates device
  * memory (tables and scratch); synchronizes the device once.
  */
@@ -240,8 +240,8 @@ eco_status eco_step_host(const eco_config* cfg, const eco_tensor* tensors, size_
  * 4096 parameters, each tensor rounded up to whole units); beyond either the call returns
  * ECO_ERR_INVALID_ARG, says so in eco_last_error(NULL), and launches nothing.
  * Behaviour to know about:
- *   - The first call on each device looks up the array's device address (with that device current).
- *     Make that first call outside any stream capture.
+ *   - The first call on each device looks up the array's device address (with that device current);
+ *     that first call should come before any stream capture.
  *   - All calls share the one array, which still holds the previous call's tables: every call
  *     rewrites what it uses and zeroes its reduction slots first.  Two calls whose GPU work overlaps
  *     (different streams, or different host threads) race on it; serialize them.

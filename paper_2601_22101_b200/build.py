@@ -9,7 +9,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(_HERE, "csrc")
 LIB = os.path.join(_HERE, "libeco_b200.so")
 SOURCES = ["eco_api.cu", "eco_kernels.cu", "eco_stream_kernels.cu"]
-HEADERS = ["eco_device.cuh", "eco_launch.h", os.path.join("..", "..", "include", "eco.h")]
+HEADERS = ["eco_device.cuh", "eco_launch.h", "eco_index.h", os.path.join("..", "..", "include", "eco.h")]
 NVCC_FLAGS = ["-O3", "-std=c++17", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",
               "-fmad=false", "-Xcompiler", "-fPIC", "-Xcompiler", "-Wall"]
 

@@ -991,6 +991,9 @@ eco_status eco_step_static(const eco_config* cfg, const eco_tensor* tensors, siz
         if (eco_status st = check_shape(*cfg, t.rows, t.cols, i)) return st;
         if ((static_cast<uint64_t>(t.row_offset) * static_cast<uint64_t>(t.cols)) % 4 != 0)
             return fail(nullptr, ECO_ERR_INVALID_ARG, "tensor %zu: row_offset * cols must be a multiple of 4", i);
+        if (static_cast<unsigned __int128>(static_cast<uint64_t>(t.row_offset) + static_cast<uint64_t>(t.rows)) *
+                static_cast<unsigned __int128>(t.cols) >= (static_cast<unsigned __int128>(1) << 34))
+            return fail(nullptr, ECO_ERR_INVALID_ARG, "tensor %zu: (row_offset + rows) * cols must be < 2^34", i);
         if (adam != (t.v != nullptr)) return fail(nullptr, ECO_ERR_INVALID_ARG, "tensor %zu: v must be given for Adam and NULL for SGDM", i);
         for (size_t j = 0; j < i; ++j)
             if (tensors[j].tensor_id == t.tensor_id) return fail(nullptr, ECO_ERR_INVALID_ARG, "tensor %zu: duplicate tensor_id %u", i, t.tensor_id);

@@ -20,6 +20,7 @@
 #include <algorithm>
 
 #include "eco_device.cuh"
+#include "eco_index.h"
 #include "eco_launch.h"
 
 namespace eco {
@@ -89,7 +90,7 @@ __device__ __forceinline__ bool scale32_index(const TensorDesc& T, uint64_t blk,
     const uint64_t row = blk / T.blocks_per_row;
     const uint32_t j = static_cast<uint32_t>(blk - row * T.blocks_per_row);
     k = row * T.scales_per_row + j * 4u + g;
-    return j * 128u + 32u * g < T.cols;
+    return block32_inside(T.cols, j, static_cast<uint32_t>(g));
 }
 
 // ---------------------------------------------------------------------------
@@ -241,10 +242,10 @@ eco_row_kernel(const TensorDesc* __restrict__ descs, const uint32_t* __restrict_
     const bool vec = (start & 3) == 0;
     const float s_old = load_scale(T.scale, row, scale_kind);
     float amax = 0.0f;
-    for (uint32_t c = 4 * threadIdx.x; c < T.cols; c += 4 * kThreads) {
-        const uint32_t rem = T.cols - c;
+    // 64-bit column counter: cols may be anything below 2^32, and c + 1024 must not wrap
+    for (uint64_t c = 4 * threadIdx.x; c < T.cols; c += 4 * kThreads) {
         Lane4<OPT> L;
-        amax = fmaxf(amax, lane_front<FMT, OPT>(T, P, start + c, rem > 4 ? 4 : static_cast<int>(rem), vec, s_old, L, false));
+        amax = fmaxf(amax, lane_front<FMT, OPT>(T, P, start + c, tile_valid(T.cols, c), vec, s_old, L, false));
     }
     amax = warp_max(amax);
     if (lane == 0) smax[warp] = amax;
@@ -262,9 +263,8 @@ eco_row_kernel(const TensorDesc* __restrict__ descs, const uint32_t* __restrict_
     }
     __syncthreads();
     const float s = s_sh, inv = inv_sh;
-    for (uint32_t c = 4 * threadIdx.x; c < T.cols; c += 4 * kThreads) {
-        const uint32_t rem = T.cols - c;
-        const int nvalid = rem > 4 ? 4 : static_cast<int>(rem);
+    for (uint64_t c = 4 * threadIdx.x; c < T.cols; c += 4 * kThreads) {
+        const int nvalid = tile_valid(T.cols, c);
         Lane4<OPT> L;
         lane_front<FMT, OPT>(T, P, start + c, nvalid, vec, s_old, L, true);
         lane_back<FMT, OPT, RND>(T, P, start + c, nvalid, vec, s, inv, L);
@@ -336,8 +336,8 @@ eco_quantize_kernel(const float* __restrict__ x, uint8_t* __restrict__ w, void* 
             const uint64_t start = row * cols;
             const bool vec = (start & 3) == 0;
             float amax = 0.0f;
-            for (uint32_t c = 4 * threadIdx.x; c < cols; c += 4 * kThreads)
-                amax = fmaxf(amax, amax_lane(x, start + c, min(4u, cols - c), vec));
+            for (uint64_t c = 4 * threadIdx.x; c < cols; c += 4 * kThreads)
+                amax = fmaxf(amax, amax_lane(x, start + c, tile_valid(cols, c), vec));
             amax = warp_max(amax);
             if (lane == 0) smax[warp] = amax;
             __syncthreads();
@@ -353,14 +353,14 @@ eco_quantize_kernel(const float* __restrict__ x, uint8_t* __restrict__ w, void* 
             }
             __syncthreads();
             const float inv = inv_sh;
-            for (uint32_t c = 4 * threadIdx.x; c < cols; c += 4 * kThreads)
-                quantize_lane<FMT, RND>(x, w, start + c, min(4u, cols - c), vec, inv, P, tensor_id);
+            for (uint64_t c = 4 * threadIdx.x; c < cols; c += 4 * kThreads)
+                quantize_lane<FMT, RND>(x, w, start + c, tile_valid(cols, c), vec, inv, P, tensor_id);
             __syncthreads();
         }
         return;
     }
     // mode 3 / 4: one warp per chunk of 128 elements of a row = one scale block (mode 3) or four of 32 (mode 4)
-    const uint32_t bpr = (cols + 127u) / 128u;
+    const uint32_t bpr = div_ceil_u32(cols, 128u);
     const uint64_t n_blocks = rows * bpr;
     for (uint64_t blk = static_cast<uint64_t>(blockIdx.x) * kWarps + warp; blk < n_blocks;
          blk += static_cast<uint64_t>(gridDim.x) * kWarps) {
@@ -377,8 +377,8 @@ eco_quantize_kernel(const float* __restrict__ x, uint8_t* __restrict__ w, void* 
         if (mode == 4) {
             make_scale<FMT>(group8_max(mine), scale_kind, s, inv, s_bits);
             const uint32_t g = static_cast<uint32_t>(lane) >> 3;
-            if ((lane & 7) == 0 && c0 + 32u * g < cols)
-                store_scale(scale, row * ((cols + 31u) / 32u) + c0 / 32u + g, scale_kind, s, s_bits);
+            if ((lane & 7) == 0 && block32_inside(cols, c0 / 128u, g))
+                store_scale(scale, row * div_ceil_u32(cols, 32u) + c0 / 32u + g, scale_kind, s, s_bits);
         } else {
             make_scale<FMT>(warp_max(mine), scale_kind, s, inv, s_bits);
             if (lane == 0) store_scale(scale, blk, scale_kind, s, s_bits);
@@ -467,7 +467,8 @@ template <int FMT, bool OUT_BF16>
 __global__ void __launch_bounds__(kThreads)
 eco_dequantize_kernel(const uint8_t* __restrict__ w, const void* __restrict__ scale, void* __restrict__ out,
                       const uint64_t rows, const uint32_t cols, const int gran, const uint32_t block, const int scale_kind) {
-    const uint32_t quads_per_row = (cols + 3u) / 4u;
+    const uint32_t quads_per_row = div_ceil_u32(cols, 4u);
+    const uint32_t scales_per_row = div_ceil_u32(cols, block);
     const uint64_t n_quads = rows * quads_per_row;
     for (uint64_t qd = static_cast<uint64_t>(blockIdx.x) * kThreads + threadIdx.x; qd < n_quads;
          qd += static_cast<uint64_t>(gridDim.x) * kThreads) {
@@ -482,7 +483,7 @@ eco_dequantize_kernel(const uint8_t* __restrict__ w, const void* __restrict__ sc
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
             if (e >= nvalid) break;
-            const uint64_t k = gran == 0 ? 0 : (gran == 1 ? row : row * ((cols + block - 1u) / block) + (c0 + e) / block);
+            const uint64_t k = gran == 0 ? 0 : (gran == 1 ? row : row * scales_per_row + (c0 + e) / block);
             const float x = __fmul_rn(val[e], load_scale(scale, k, scale_kind));
             if (OUT_BF16) static_cast<uint16_t*>(out)[i0 + e] = static_cast<uint16_t>(f32_to_bf16_bits_rne(x));
             else static_cast<float*>(out)[i0 + e] = x;
@@ -496,13 +497,18 @@ eco_dequantize_kernel(const uint8_t* __restrict__ w, const void* __restrict__ sc
 template <int FMT, bool OUT_BF16, int EPT>
 __global__ void __launch_bounds__(kThreads)
 eco_dequantize_vec_kernel(const uint8_t* __restrict__ w, const void* __restrict__ scale, void* __restrict__ out,
-                          const uint32_t n_units, const uint32_t units_per_row, const int gran, const uint32_t block,
+                          const uint64_t n_units, const uint32_t units_per_row, const int gran, const uint32_t block,
                           const uint32_t scales_per_row, const int scale_kind) {
     static_assert(EPT == 4 || EPT == 8, "4 or 8 elements per thread");
     constexpr int Q = EPT / 4;
-    for (uint32_t u = blockIdx.x * kThreads + threadIdx.x; u < n_units; u += gridDim.x * kThreads) {
-        const uint32_t row = u / units_per_row, c0 = (u - row * units_per_row) * EPT;
-        const uint64_t i0 = static_cast<uint64_t>(u) * EPT;
+    // 64-bit unit counter and stride: n_units reaches 2^32 - 4 for the largest admitted tensor, and u + stride
+    // must not wrap below it
+    for (uint64_t u = static_cast<uint64_t>(blockIdx.x) * kThreads + threadIdx.x; u < n_units;
+         u += static_cast<uint64_t>(gridDim.x) * kThreads) {
+        uint64_t row;
+        uint32_t c0;
+        dequant_unit_position(u, units_per_row, EPT, row, c0);
+        const uint64_t i0 = u * EPT;
         uint32_t codes[Q];
         if (FMT != FMT_INT4) {
             if constexpr (EPT == 8) {
@@ -519,7 +525,7 @@ eco_dequantize_vec_kernel(const uint8_t* __restrict__ w, const void* __restrict_
                 codes[0] = __ldg(reinterpret_cast<const uint16_t*>(w + (i0 >> 1)));
             }
         }
-        const uint64_t k = gran == 0 ? 0 : (gran == 1 ? row : static_cast<uint64_t>(row) * scales_per_row + c0 / block);
+        const uint64_t k = gran == 0 ? 0 : (gran == 1 ? row : row * scales_per_row + c0 / block);
         const float s = load_scale(scale, k, scale_kind);
         float x[EPT];
 #pragma unroll
@@ -550,11 +556,11 @@ cudaError_t launch_dequantize(const LaunchConfig& c, const uint8_t* w, const voi
     const uint32_t block = static_cast<uint32_t>(128 / c.sub);
     const bool aligned = ((reinterpret_cast<uintptr_t>(w) | reinterpret_cast<uintptr_t>(out)) & 15u) == 0;
     if (cols % 16 == 0 && aligned) {
-        const uint32_t ept = out_bf16 ? 8u : 4u;                       // rows * cols < 2^34: unit indices fit 32 bits
-        const uint32_t n_units = static_cast<uint32_t>(rows * cols / ept);
-        const uint32_t cap = static_cast<uint32_t>((c.sm_count > 0 ? c.sm_count : 148) * 16);
-        const uint32_t g = std::max(1u, std::min(cap, (n_units + kThreads - 1) / kThreads));
-        const uint32_t spr = (cols + block - 1) / block;
+        const uint32_t ept = out_bf16 ? 8u : 4u;
+        const uint64_t n_units = dequant_units(rows, cols, ept);
+        const uint64_t cap = static_cast<uint64_t>((c.sm_count > 0 ? c.sm_count : 148) * 16);
+        const uint32_t g = static_cast<uint32_t>(std::max<uint64_t>(1, std::min(cap, (n_units + kThreads - 1) / kThreads)));
+        const uint32_t spr = div_ceil_u32(cols, block);
         ECO_DISPATCH_FMT(c.format, {
             if (out_bf16) eco_dequantize_vec_kernel<F, true, 8><<<g, kThreads, 0, stream>>>(w, scale, out, n_units, cols / 8, gran, block, spr, c.scale_kind);
             else eco_dequantize_vec_kernel<F, false, 4><<<g, kThreads, 0, stream>>>(w, scale, out, n_units, cols / 4, gran, block, spr, c.scale_kind);

@@ -18,6 +18,7 @@
 // waiter records a code in the context's status word and leaves; the producer
 // first waits (bounded again) for the copies it has in flight.
 #include "eco_device.cuh"
+#include "eco_index.h"
 #include "eco_launch.h"
 
 namespace eco {
@@ -378,8 +379,8 @@ eco_stream_kernel(const TensorDesc* __restrict__ descs, const uint32_t* __restri
         // mixes compute-heavy and memory-heavy tensors on every SM.  tickets[0] counts tickets, tickets[1] CTAs
         // that are done drawing; the last one rewinds both for the next launch.
         const uint32_t W = static_cast<uint32_t>(interleave);
-        const uint32_t per_region = (n_units + W - 1) / W;
-        const uint32_t n_tickets = per_region * W;
+        const uint32_t per_region = div_ceil_u32(n_units, W);
+        const uint32_t n_tickets = ticket_count(n_units, W);   // n_units < 2^31: fits, with room for the draws past the end
         auto draw = [&]() -> uint32_t {
             uint32_t t = 0;
             if (lane == 0) t = atomicAdd(tickets, 1u);
