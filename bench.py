@@ -6,8 +6,13 @@
 One "step" is one eco_step over every tensor of the workload's parameter set (the whole hot path:
 dequantize, optimizer update, amax/scale, requantize with stochastic rounding, error injection, stores).
 Prints ONE JSON line.  `value` = parameters updated per second with the state resident in HBM, timed
-with CUDA events on the launching stream; `e2e` = the same metric through eco_host_step with the state
-in pinned HOST memory (copies inside the timed region).  With torchrun (N > 1) every rank steps its own
+with CUDA events on the launching stream: blocks of exactly --steps steps, each bracketed by a barrier and
+a synchronize, repeated until at least --min-seconds have been timed so that the GPU reaches the clock its
+power cap allows; `value` is the MEDIAN block, the first block is reported beside it.  The default workload
+is the largest of the benchmark sets that fits one GPU (c5, 15.5 B parameters); the other sets of a billion
+parameters or more are timed after it and `roofline.min_frac_1b_plus` is the smallest of their fractions.
+`e2e` = the same metric through eco_host_step with the state in pinned HOST memory (copies inside the
+timed region).  With torchrun (N > 1) every rank steps its own
 replica of the parameter set (no data-path collective exists in this method) and the time is the max
 over ranks.  `--impl reference` times the CPU oracle instead (rank 0 only).
 """
@@ -27,20 +32,44 @@ if ROOT not in sys.path:
 METRIC = "eco_optimizer_step_params_per_sec"
 UNIT = "params/s"
 FALLBACK_HBM_GBS = 6650.0
+# the benchmark sets of a billion parameters or more, as configured
+BIG_SETS = ("c3_gemma3_1b_fp8_tensor_adam_sr", "c4_smoe_2mat_fp8_block128_adam_sr", "c5_deepseek_moe16b_int4_group128_sgdm_sr")
 
-# DRAM traffic per parameter of the dominant kernel from an ncu capture
-# (dram__bytes_read.sum + dram__bytes_write.sum over the launch, divided by its parameters);
-# sources are the summaries under profiles/.  None = not captured.
-NCU_DRAM_BYTES_PER_PARAM = {
-    # profiles/eco_stream_kernel_c4s.md: 1.4808 GB read + 1.1625 GB written over 134,217,728 parameters
-    "eco_stream_kernel<fp8,adam,sr,block>": 19.69,
-    # profiles/eco_stream_kernel_c5s.md: 1.1941 GB + 0.7726 GB over 183,304,192 parameters
-    "eco_stream_kernel<int4,sgdm,sr,block>": 10.73,
-    # profiles/eco_stream_kernel_c3s.md (apply pass): 1.0058 GB + 0.7683 GB over 91,422,720 parameters
-    "eco_stream_kernel<fp8,adam,sr,tensor_apply>": 19.41,
-    # profiles/eco_stream_kernel_c4mxs.md: 1.4812 GB + 1.1603 GB over 134,217,728 parameters
-    "eco_stream_kernel<fp8,adam,sr,block32>": 19.68,
-}
+PROFILE_SOURCES = ("eco_stream_kernels.cu", "eco_device.cuh", "eco_index.h")
+
+
+def _kernel_sources_digest() -> str:
+    """SHA-256 over the sources the streaming kernels are built from: an ncu summary carries the digest of the
+    sources it was captured on, and its counters are not quoted once they have changed."""
+    import hashlib
+    h = hashlib.sha256()
+    for name in PROFILE_SOURCES:
+        with open(os.path.join(ROOT, "paper_2601_22101_b200", "csrc", name), "rb") as f:
+            h.update(f.read())
+    return h.hexdigest()
+
+
+def _ncu_dram_bytes_per_param():
+    """DRAM bytes per parameter (dram__bytes_read.sum + dram__bytes_write.sum over a launch, divided by its
+    parameters) of every streaming-kernel instantiation that has a tracked ncu summary, read from the summaries at
+    run time: {"<template arguments>": B/param}.  A summary whose source digest differs from the current sources is
+    skipped (the kernel changed since the counters were taken)."""
+    import glob
+    import re
+    out = {}
+    digest = _kernel_sources_digest()
+    for path in sorted(glob.glob(os.path.join(ROOT, "profiles", "eco_stream_kernel_*.md"))):
+        text = open(path).read()
+        m = re.search(r"kernel sources sha256: ([0-9a-f]{64})", text)
+        if not m or m.group(1) != digest:
+            continue
+        for sec in text.split("\n## ")[1:]:
+            name = sec.split("\n", 1)[0].strip()
+            k = re.match(r"eco_stream_kernel<([0-9, ]+)>", name)
+            v = re.search(r"derived: DRAM bytes per parameter \| ([0-9.]+) B", sec)
+            if k and v:
+                out.setdefault(k.group(1).replace(" ", ""), []).append(float(v.group(1)))
+    return {k: sum(v) / len(v) for k, v in out.items()}
 
 
 def _workload(name: str):
@@ -48,15 +77,24 @@ def _workload(name: str):
     return wl.BY_NAME[name]()
 
 
-def _dominant_kernel(w) -> str:
-    """Name of the kernel that moves most of a step's bytes (full-size sets are made of whole 128-element rows,
-    which the persistent TMA-fed kernel takes)."""
+def _dominant_kernel(w):
+    """(readable name, template arguments of its launches) of the kernel that moves most of a step's bytes: full-size
+    sets are made of whole 128-element rows, which the persistent TMA-fed kernel takes.  Per-tensor scales are a
+    pair of launches (amax pass, apply pass)."""
     from paper_2601_22101_b200 import workloads as wl
     fmt = {wl.FP8_E4M3: "fp8", wl.INT4: "int4", wl.FP8_E5M2: "e5m2"}[w.format]
+    fi = {wl.FP8_E4M3: 0, wl.INT4: 1, wl.FP8_E5M2: 2}[w.format]
     opt = "adam" if w.optimizer == wl.ADAM else "sgdm"
+    oi = 1 if w.optimizer == wl.ADAM else 0
     rnd = "sr" if w.rounding == wl.SR else "rtn"
+    ri = 1 if w.rounding == wl.SR else 0
     mode = {wl.PER_BLOCK: "block" if w.block == 128 else "block32", wl.PER_TENSOR: "tensor_apply", wl.PER_ROW: "row"}[w.granularity]
-    return f"eco_stream_kernel<{fmt},{opt},{rnd},{mode}>"
+    if w.granularity == wl.PER_TENSOR:
+        args = [f"{fi},{oi},0,1,0", f"{fi},{oi},{ri},2,0"]
+    else:
+        mi = {"block": 0, "row": 3, "block32": 4}[mode]
+        args = [f"{fi},{oi},{ri},{mi},0"]
+    return f"eco_stream_kernel<{fmt},{opt},{rnd},{mode}>", args
 
 
 def _two_pass_note(w, params, ms_per_step, peak):
@@ -267,27 +305,30 @@ def run_e2e(w, device: int, steps: int, max_host_gb: float):
     return {"value": ws.numel * steps / el, "unit": UNIT, "h2d_bytes_per_step": up, "d2h_bytes_per_step": down,
             "h2d_copies_per_step": n_in, "d2h_copies_per_step": n_out,
             "steps": steps, "params_per_step": ws.numel, "seconds": el,
-            "sample": f"first {len(picked)} of {len(w.tensors)} tensors per GPU held in pinned host memory"}
+            "sample": f"first {len(picked)} of {len(w.tensors)} tensors per GPU ({ws.numel / w.numel:.1%} of the parameters) "
+                      f"held in pinned host memory"}
 
 
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=5)
-    ap.add_argument("--workload", default="c4", choices=["c1", "c2", "c3", "c4", "c5", "c3r", "c5t", "c4g", "c4d", "c3s", "c3rs", "c4s", "c5s", "c4mx", "c4mxs", "c4ds"])
+    ap.add_argument("--workload", default="c5", choices=["c1", "c2", "c3", "c4", "c5", "c3r", "c5t", "c4g", "c4d", "c3s", "c3rs", "c4s", "c5s", "c4mx", "c4mxs", "c4ds"])
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--also", default="c3,c5,c4mx", help="comma-separated workloads timed after the headline one and "
+    ap.add_argument("--min-seconds", type=float, default=2.0, help="blocks of --steps steps are repeated until this much has been timed")
+    ap.add_argument("--also", default="c3,c4,c4d", help="comma-separated workloads timed after the headline one and "
                     "reported under other_workloads (device-resident timing only)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--e2e-steps", type=int, default=5)
-    ap.add_argument("--e2e-host-gb", type=float, default=8.0)
+    ap.add_argument("--e2e-host-gb", type=float, default=24.0, help="pinned host memory the end-to-end leg may hold; the "
+                    "leg runs on the first tensors of the set that fit and says which fraction that was")
     ap.add_argument("--option", action="append", default=[], help="name=value passed to eco_set_option")
     args = ap.parse_args()
 
     if args.impl == "reference":
-        if args.steps == 100 and args.warmup == 5:
+        if args.steps == 20 and args.warmup == 5:
             args.steps, args.warmup = 5, 1
         run_reference(args)
         return
@@ -310,8 +351,12 @@ def main():
         k, v = o.split("=")
         eco.eco_set_option(k, int(v))
 
-    def time_workload(w_global, steps, warmup, sample_clocks):
-        """Device-resident timing of `steps` eco_steps of this rank's shard; returns a dict (rank 0) or None."""
+    ncu_bpp = _ncu_dram_bytes_per_param()
+
+    def time_workload(w_global, steps, warmup, min_seconds):
+        """Device-resident timing of this rank's shard: blocks of `steps` eco_steps, each bracketed by a barrier and a
+        synchronize and timed with CUDA events on the launching stream (max over ranks), repeated until min_seconds
+        have been timed.  Returns a dict (rank 0) or None."""
         w_rank = wl.shard(wl.replicate(w_global, world), rank, world) if world > 1 else w_global
         st = DeviceState(w_rank, local)
         st.init_on_device(seed=1234 + rank)
@@ -323,45 +368,59 @@ def main():
             step_no += 1
             st.step(step_no, stream.cuda_stream)
         barrier()
-        sampler = ClockSampler(local) if sample_clocks else None
-        if sampler:
-            sampler.start()
-        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        ev0.record(stream)
-        for _ in range(steps):
-            step_no += 1
-            st.step(step_no, stream.cuda_stream)
-        ev1.record(stream)
-        barrier()
-        clocks = sampler.stop() if sampler else None
+        sampler = ClockSampler(local)
+        sampler.start()
+        blocks, total_ms = [], 0.0
+        while True:
+            ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            ev0.record(stream)
+            for _ in range(steps):
+                step_no += 1
+                st.step(step_no, stream.cuda_stream)
+            ev1.record(stream)
+            barrier()
+            ms = ev0.elapsed_time(ev1)
+            if world > 1:
+                t = torch.tensor([ms], device="cuda", dtype=torch.float64)
+                dist.all_reduce(t, op=dist.ReduceOp.MAX)
+                ms = float(t.item())
+            blocks.append(ms / steps)
+            total_ms += ms
+            if total_ms >= min_seconds * 1e3 or len(blocks) >= 200:     # same decision on every rank (ms is reduced)
+                break
+        clocks = sampler.stop()
         eco.eco_check(st.handle, stream.cuda_stream)
-        ms = ev0.elapsed_time(ev1)
-        if world > 1:
-            t = torch.tensor([ms], device="cuda", dtype=torch.float64)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms = float(t.item())
-        ms_per_step = ms / steps
         state_bytes = st.device_bytes()
         st.destroy()
         del st
         torch.cuda.empty_cache()
         if rank != 0:
             return None
+        ms_per_step = sorted(blocks)[len(blocks) // 2]
         peak, peak_src = _measured_peak()
         bpp = w_global.algorithmic_bytes_per_param()
         params_per_rank = w_rank.numel
-        achieved = params_per_rank * bpp / (ms_per_step * 1e-3) / 1e9
-        kern = _dominant_kernel(w_global)
-        tr = NCU_DRAM_BYTES_PER_PARAM.get(kern)
+        gbs = lambda ms: params_per_rank * bpp / (ms * 1e-3) / 1e9
+        achieved = gbs(ms_per_step)
+        kern, targs = _dominant_kernel(w_global)
+        tr = sum(ncu_bpp[a] for a in targs) if all(a in ncu_bpp for a in targs) else None
+        mhz = clocks.get("sm_mhz") if clocks else None
         return {
             "workload": w_global.name, "params_per_gpu": params_per_rank, "tensors_per_gpu": len(w_rank.tensors),
             "ms_per_step": ms_per_step, "value": params_per_rank * world / (ms_per_step * 1e-3),
+            "blocks": len(blocks), "steps_per_block": steps, "timed_seconds": total_ms * 1e-3,
+            "first_block": {"ms_per_step": blocks[0], "value": params_per_rank * world / (blocks[0] * 1e-3),
+                            "frac": gbs(blocks[0]) / peak},
+            "ms_per_step_x_sm_mhz": (ms_per_step * mhz if mhz else None),
             "launches_per_step": launches_per_step, "state_bytes_on_device": state_bytes, "clocks": clocks,
             "roofline": {"bound": "hbm", "kernel": kern, "achieved": achieved, "peak": peak, "unit": "GB/s",
                          "frac": achieved / peak, "peak_source": peak_src,
                          "frac_of_nominal_8000": achieved / 8000.0,
                          "algorithmic_bytes_per_param": bpp,
                          "traffic": (tr * params_per_rank if tr else None),
+                         "traffic_source": ("ncu DRAM bytes per parameter of this kernel on the small capture case "
+                                            "(profiles/), times the parameters of a full launch" if tr else
+                                            "no ncu summary taken on the current kernel sources"),
                          **_two_pass_note(w_global, params_per_rank, ms_per_step, peak)},
         }
 
@@ -374,15 +433,23 @@ def main():
         torch.cuda.synchronize()
 
     w = _workload(args.workload)
-    head = time_workload(w, args.steps, args.warmup, True)
+    head = time_workload(w, args.steps, args.warmup, args.min_seconds)
     others = []
     for name in [n for n in args.also.split(",") if n and n != args.workload]:
-        r = time_workload(_workload(name), min(args.steps, 20), 3, True)
+        r = time_workload(_workload(name), args.steps, 3, args.min_seconds)
         if r is not None:
-            others.append({k: r[k] for k in ("workload", "params_per_gpu", "ms_per_step", "value", "launches_per_step",
-                                             "clocks", "roofline")})
+            others.append({k: r[k] for k in ("workload", "params_per_gpu", "ms_per_step", "value", "blocks", "first_block",
+                                             "ms_per_step_x_sm_mhz", "launches_per_step", "clocks", "roofline")})
 
     if rank == 0:
+        # the benchmark sets of a billion parameters or more, as configured (c3, c4, c5): the smallest fraction of the roofline
+        big = [r for r in [head] + others if r["workload"] in BIG_SETS]
+        roof = dict(head["roofline"])
+        if big:
+            worst = min(big, key=lambda r: r["roofline"]["frac"])
+            roof["min_frac_1b_plus"] = worst["roofline"]["frac"]
+            roof["min_frac_1b_plus_workload"] = worst["workload"]
+            roof["fracs_1b_plus"] = {r["workload"]: r["roofline"]["frac"] for r in big}
         out = {
             "metric": METRIC, "value": head["value"], "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": head["ms_per_step"], "higher_is_better": True,
@@ -390,11 +457,15 @@ def main():
             "config": {"workload": w.name, "params_per_gpu": head["params_per_gpu"],
                        "tensors_per_gpu": head["tensors_per_gpu"],
                        "state_bytes_on_device": head["state_bytes_on_device"],
+                       "timing": f"blocks of {args.steps} steps (barrier + synchronize on both sides, CUDA events on the "
+                                 f"launching stream) repeated until {args.min_seconds} s were timed; value = median block",
                        "l2": "inputs much larger than the 126 MB L2, streamed once per step (no flush needed)",
                        "sharding": "whole tensors per rank, no data-path collective" if world > 1 else "single GPU"},
-            "gpu_launches": head["launches_per_step"] * args.steps,
+            "blocks": head["blocks"], "timed_seconds": head["timed_seconds"], "first_block": head["first_block"],
+            "ms_per_step_x_sm_mhz": head["ms_per_step_x_sm_mhz"],
+            "gpu_launches": head["launches_per_step"] * args.steps * head["blocks"],
             "clocks": head["clocks"],
-            "roofline": head["roofline"],
+            "roofline": roof,
             "other_workloads": others,
         }
     if not args.no_e2e:

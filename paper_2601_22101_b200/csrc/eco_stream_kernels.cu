@@ -112,11 +112,12 @@ __device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_
 }
 
 // max |x| over the 32 lanes in one instruction (sm_100a warp reduction on binary32; NaN operands are
-// ignored, as by fmaxf).  Every lane receives the result.
+// ignored, as by fmaxf).  Every lane receives the result.  The final maximum with zero makes a warp whose
+// operands are ALL NaN return 0 (a block of nothing but NaN has no maximum: it takes the scale of an all-zero block).
 __device__ __forceinline__ float warp_amax(float x) {
     float r;
     asm volatile("redux.sync.max.abs.f32 %0, %1, 0xffffffff;" : "=f"(r) : "f"(x));
-    return r;
+    return fmaxf(r, 0.0f);
 }
 
 __device__ __forceinline__ uint32_t units_of(const TensorDesc& T) {
@@ -246,7 +247,7 @@ __device__ __forceinline__ bool consume_unit(const StepParams& P, const int scal
         const float x = fmaxf(b2 ? amax[2] : amax[0], __shfl_xor_sync(0xFFFFFFFFu, b2 ? amax[0] : amax[2], 4));
         const float y = fmaxf(b2 ? amax[3] : amax[1], __shfl_xor_sync(0xFFFFFFFFu, b2 ? amax[1] : amax[3], 4));
         float z = fmaxf(b1 ? y : x, __shfl_xor_sync(0xFFFFFFFFu, b1 ? x : y, 2));
-        z = fmaxf(z, __shfl_xor_sync(0xFFFFFFFFu, z, 1));
+        z = fmaxf(fmaxf(z, __shfl_xor_sync(0xFFFFFFFFu, z, 1)), 0.0f);     // (an all-NaN block: 0, like warp_amax)
         const int rr = (lane >> 1) & 3, g8 = lane >> 3;
         float s_mine, inv_mine;
         uint32_t bits_mine;

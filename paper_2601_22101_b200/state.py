@@ -16,14 +16,28 @@ from . import eco
 from . import workloads as wl
 
 _ALIGN = 256
+_GUARD = 256          # bytes of guard before the first view, between views and after the last
+_SENTINEL = 0xA5
 
 
 def _carve(sizes_bytes: List[int]):
-    offs, total = [], 0
+    """Offsets of the views inside one allocation: every view starts on a 256-byte boundary and is preceded and
+    followed by at least _GUARD bytes that belong to no tensor (the guard areas, see DeviceState.check_guards)."""
+    offs, total = [], _GUARD
     for b in sizes_bytes:
         offs.append(total)
-        total += (b + _ALIGN - 1) // _ALIGN * _ALIGN
-    return offs, max(total, _ALIGN)
+        total += (b + _ALIGN - 1) // _ALIGN * _ALIGN + _GUARD
+    return offs, total
+
+
+def _guard_index(offs: List[int], sizes_bytes: List[int], total: int, device) -> torch.Tensor:
+    """Byte positions of an allocation that lie in no view (int64 tensor on the device)."""
+    starts = torch.tensor([0] + [o + b for o, b in zip(offs, sizes_bytes)], dtype=torch.int64)
+    ends = torch.tensor(offs + [total], dtype=torch.int64)
+    lens = ends - starts
+    first = torch.repeat_interleave(starts, lens)
+    within = torch.arange(int(lens.sum()), dtype=torch.int64) - torch.repeat_interleave(torch.cumsum(lens, 0) - lens, lens)
+    return (first + within).to(device)
 
 
 def config_of(w: wl.Workload, injection: int = eco.ECO_INJECT_ECO) -> eco.Config:
@@ -43,15 +57,28 @@ class DeviceState:
         ts = w.tensors
         adam = w.optimizer == wl.ADAM
         sb = wl.SCALE_BYTES[w.scale_dtype]
-        self._w_off, w_total = _carve([w.code_bytes(t) for t in ts])
-        self._s_off, s_total = _carve([w.n_scales(t) * sb for t in ts])
-        self._g_off, g_total = _carve([t.numel * 2 for t in ts])
-        self._m_off, m_total = _carve([t.numel * 4 for t in ts])
+        w_sizes, s_sizes = [w.code_bytes(t) for t in ts], [w.n_scales(t) * sb for t in ts]
+        g_sizes, m_sizes = [t.numel * 2 for t in ts], [t.numel * 4 for t in ts]
+        self._w_off, w_total = _carve(w_sizes)
+        self._s_off, s_total = _carve(s_sizes)
+        self._g_off, g_total = _carve(g_sizes)
+        self._m_off, m_total = _carve(m_sizes)
         self.w_buf = torch.zeros(w_total, dtype=torch.uint8, device=dev)
         self.s_buf = torch.zeros(s_total, dtype=torch.uint8, device=dev)
         self.g_buf = torch.zeros(g_total, dtype=torch.uint8, device=dev)
         self.m_buf = torch.zeros(m_total, dtype=torch.uint8, device=dev)
         self.v_buf = torch.zeros(m_total, dtype=torch.uint8, device=dev) if adam else None
+        # Guard areas: every byte of the five allocations that belongs to no tensor holds a sentinel.  A kernel that
+        # stores past the end of a ragged tensor (or before its start) changes one, and check_guards() sees it.
+        self._guards = []
+        for buf, offs, sizes, total in ((self.w_buf, self._w_off, w_sizes, w_total), (self.s_buf, self._s_off, s_sizes, s_total),
+                                        (self.g_buf, self._g_off, g_sizes, g_total), (self.m_buf, self._m_off, m_sizes, m_total),
+                                        (self.v_buf, self._m_off, m_sizes, m_total)):
+            if buf is None:
+                continue
+            idx = _guard_index(offs, sizes, total, dev)
+            buf[idx] = _SENTINEL
+            self._guards.append((buf, idx))
         self.tensors: List[eco.Tensor] = []
         sdt = {wl.SCALE_F32: torch.float32, wl.SCALE_BF16: torch.bfloat16, wl.SCALE_E8M0: torch.uint8}[w.scale_dtype]
         for i, t in enumerate(ts):
@@ -126,6 +153,19 @@ class DeviceState:
         if self.handle is not None:
             eco.eco_destroy(self.handle)
             self.handle = None
+
+    def check_guards(self) -> None:
+        """Raise if any byte outside the tensors' views was written since construction."""
+        names = ("codes", "scales", "gradients", "m", "v")
+        for name, (buf, idx) in zip(names, self._guards):
+            got = buf[idx]
+            if not bool((got == _SENTINEL).all()):
+                bad = idx[got != _SENTINEL]
+                raise AssertionError(f"guard bytes of the {name} allocation were overwritten: {bad.numel()} bytes, "
+                                     f"first at offset {int(bad[0])}")
+
+    def guard_bytes(self) -> int:
+        return sum(int(idx.numel()) for _, idx in self._guards)
 
     def device_bytes(self) -> int:
         return sum(b.numel() for b in (self.w_buf, self.s_buf, self.g_buf, self.m_buf, self.v_buf) if b is not None)

@@ -37,6 +37,7 @@ STRICT_MOMENTS = False      # set by test_moments_match_bit_for_bit: m and v com
 
 
 def compare(dev: DeviceState, ora: OracleState, where=""):
+    dev.check_guards()                       # no kernel wrote outside the tensors' views
     for i, t in enumerate(dev.workload.tensors):
         d = dev.tensors[i]
         tag = f"{where} tensor {i} {t.name} [{t.rows}x{t.cols}]"
@@ -346,6 +347,7 @@ def _sampled_full_size(w: wl.Workload, sample_ids, steps=2):
             dev.step(step)
         torch.cuda.synchronize()
         eco.eco_check(dev.handle, torch.cuda.current_stream().cuda_stream)
+        dev.check_guards()
         for i in sample_ids:
             t = w.tensors[i]
             cw, cs, cg, cm, cv = before[i]
@@ -386,7 +388,7 @@ def test_c3_full_size_sampled_tensors():
     w = wl.c3()
     n = len(w.tensors)
     ids = list(range(7)) + list(range(n - 8, n - 1)) + [n - 1]        # first and last layer, and the 302M-parameter embedding
-    _sampled_full_size(w, ids, steps=1)
+    _sampled_full_size(w, ids, steps=2)
 
 
 def test_c5_full_size_sampled_tensors():
@@ -449,6 +451,7 @@ def test_row_shards_with_amax_exchange_equal_the_unsplit_step(fmt, opt, sdt):
     full = DeviceState(w)
     full.init_from_host()
     full.create()
+    ora = OracleState(w)                  # the oracle steps the whole, unsplit tensors
     adam = opt == wl.ADAM
     shards = []          # per rank: (tensors, handle)
     cuts = [t.rows // 2 for t in w.tensors]
@@ -471,6 +474,7 @@ def test_row_shards_with_amax_exchange_equal_the_unsplit_step(fmt, opt, sdt):
                     r0, r1 = (0, cuts[i]) if rank == 0 else (cuts[i], spec.rows)
                     ts[i].grad.copy_(d.grad[r0 * spec.cols: r1 * spec.cols])
             full.step(step, weight_decay=0.05)
+            ora.step(step, weight_decay=0.05)
             for _, h in shards:
                 eco.eco_step_begin(h, w.lr, w.beta1, w.beta2, w.eps, step, w.step_seed, 0.05, 1.0, stream)
             a0, a1 = eco.eco_amax_tensor(shards[0][1]), eco.eco_amax_tensor(shards[1][1])
@@ -483,8 +487,16 @@ def test_row_shards_with_amax_exchange_equal_the_unsplit_step(fmt, opt, sdt):
             for _, h in shards:
                 eco.eco_step_end(h, stream)
             torch.cuda.synchronize()
+            compare(full, ora, f"unsplit, step {step}")
             for i, (spec, d) in enumerate(zip(w.tensors, full.tensors)):
                 a, b = shards[0][0][i], shards[1][0][i]
+                # both shards against the oracle's whole tensor, bit for bit ...
+                assert (_np(torch.cat([a.w, b.w])) == ora.w[i]).all(), f"step {step} tensor {i}: shard codes vs oracle"
+                assert (_scale_bits(a.scale) == _oracle_scale_bits(ora.scale[i])).all(), f"step {step} tensor {i}: shard scale vs oracle"
+                assert (_np(torch.cat([a.m, b.m])).view(np.int32) == ora.m[i].view(np.int32)).all(), f"step {step} tensor {i}: shard m vs oracle"
+                if adam:
+                    assert (_np(torch.cat([a.v, b.v])).view(np.int32) == ora.v[i].view(np.int32)).all()
+                # ... and against the unsplit CUDA step
                 assert torch.equal(torch.cat([a.w, b.w]), d.w), f"step {step} tensor {i}: codes"
                 assert (_scale_bits(a.scale) == _scale_bits(d.scale)).all() and torch.equal(a.scale, b.scale)
                 assert torch.equal(torch.cat([a.m, b.m]), d.m), f"step {step} tensor {i}: m"
@@ -687,10 +699,9 @@ def test_moments_match_bit_for_bit(fmt, sdt, opt, gran, monkeypatch):
 
 def test_tensor_with_more_than_2_to_the_32_elements():
     """One tensor of 2^32 + 2^20 elements (INT4, group-128 bf16 scales, momentum SGD, stochastic rounding; 28 GB of
-    state): element offsets and the random-stream counters need more than 32 bits.  Checked on row slices: the first
-    rows against the oracle (their global indices are local ones), and rows on both sides of element 2^32 and the last
-    rows against a small context over a COPY of the slice with row_offset set, whose own arithmetic stays below 2^32
-    (that form is held to the oracle by test_row_shards_with_amax_exchange_equal_the_unsplit_step)."""
+    state): element offsets and the random-stream counters need more than 32 bits.  Checked on row slices -- the first
+    rows, rows on both sides of element 2^32 and the last rows -- against the oracle stepping a copy of the slice with
+    its position in the whole tensor, and against a small CUDA context over a copy of the slice with row_offset set."""
     rows, cols = (1 << 22) + 1024, 1024
     spec = wl.TensorSpec("huge", rows, cols, 7)
     w = wl.Workload("huge_int4", wl.INT4, wl.PER_BLOCK, 128, wl.SCALE_BF16, wl.SGDM, wl.SR, lr=5e-2, beta1=0.9, beta2=0.95,
@@ -727,14 +738,135 @@ def test_tensor_with_more_than_2_to_the_32_elements():
             assert torch.equal(shard.scale.view(torch.int16), d.scale[r0 * 8: r1 * 8].view(torch.int16)), f"rows {r0}..{r1}: scales"
             assert torch.equal(shard.m, d.m[e0: e1]), f"rows {r0}..{r1}: m"
             assert not torch.equal(shard.w, bw)                                        # the step did change the codes
-        # first rows against the oracle
-        bw, bs, bg, bm = before[0]
-        cw, cs = _np(bw).copy(), _np(bs.view(torch.int16)).view(np.uint16).copy()
-        cg, cm = _np(bg.view(torch.int16)).view(np.uint16).copy(), _np(bm).copy()
-        oracle.step(oracle_config(w), lr=float(np.float32(w.lr)), beta1=float(np.float32(w.beta1)), beta2=float(np.float32(w.beta2)),
-                    eps=float(np.float32(w.eps)), step=1, seed=w.step_seed, w=cw, scale=cs, grad=cg, m=cm, v=None,
-                    rows=8, cols=cols, tensor_id=spec.tensor_id)
-        assert (_np(d.w[: 8 * cols // 2]) == cw).all() and (_np(d.scale[: 64].view(torch.int16)).view(np.uint16) == cs).all()
-        assert (_np(d.m[: 8 * cols]).view(np.int32) == cm.view(np.int32)).all()
+        # every slice against the ORACLE, which is told where the slice sits in the whole tensor (index_base): the rows
+        # beyond element 2^32 and the last rows draw the random words of their 64-bit positions
+        for (r0, r1), (bw, bs, bg, bm) in zip(slices, before):
+            e0, e1 = r0 * cols, r1 * cols
+            cw, cs = _np(bw).copy(), _np(bs.view(torch.int16)).view(np.uint16).copy()
+            cg, cm = _np(bg.view(torch.int16)).view(np.uint16).copy(), _np(bm).copy()
+            oracle.step(oracle_config(w), lr=float(np.float32(w.lr)), beta1=float(np.float32(w.beta1)), beta2=float(np.float32(w.beta2)),
+                        eps=float(np.float32(w.eps)), step=1, seed=w.step_seed, w=cw, scale=cs, grad=cg, m=cm, v=None,
+                        rows=r1 - r0, cols=cols, tensor_id=spec.tensor_id, index_base=e0)
+            assert (_np(d.w[e0 // 2: e1 // 2]) == cw).all(), f"rows {r0}..{r1}: codes vs oracle"
+            assert (_np(d.scale[r0 * 8: r1 * 8].view(torch.int16)).view(np.uint16) == cs).all(), f"rows {r0}..{r1}: scales vs oracle"
+            assert (_np(d.m[e0: e1]).view(np.int32) == cm.view(np.int32)).all(), f"rows {r0}..{r1}: m vs oracle"
+        dev.check_guards()
     finally:
         dev.destroy()
+
+
+@pytest.mark.parametrize("fmt,sdt,opt,gran", [(wl.FP8_E4M3, wl.SCALE_F32, wl.ADAM, wl.PER_BLOCK),
+                                              (wl.FP8_E4M3, wl.SCALE_F32, wl.ADAM, wl.PER_TENSOR),
+                                              (wl.FP8_E4M3, wl.SCALE_F32, wl.ADAM, wl.PER_ROW),
+                                              (wl.INT4, wl.SCALE_BF16, wl.SGDM, wl.PER_BLOCK)])
+def test_non_finite_gradients_stay_where_they_are(fmt, sdt, opt, gran):
+    """Inf and NaN gradients (a routine event in low-precision training): the element they hit ends as NaN in the
+    moments and takes the code +rho (a NaN has no sign; block maxima ignore NaN), on both sides alike; every
+    other element -- of the same 16-element thread tile, the same scale block, the same tensor -- stays bit-exact."""
+    shapes = [(40, 512), (3, 384), (5, 200), (33, 1024)]
+    w = _mini(fmt, gran, sdt, opt, wl.SR, shapes)
+    dev = DeviceState(w)
+    dev.init_from_host()
+    ora = OracleState(w)
+    dev.create()
+    special = np.array([0x7F80, 0xFF80, 0x7FC0, 0xFFC0, 0x7FFF], np.uint16)      # +Inf, -Inf, NaN, -NaN, NaN
+    try:
+        for step in (1, 2, 3):
+            grads = [wl.gradient_bf16(w, t, step) for t in w.tensors]
+            if step == 2:
+                for i, g in enumerate(grads):
+                    pos = (np.arange(special.size) * 977 + 13 * i) % g.size      # scattered, different thread tiles
+                    g[pos] = special
+                    if g.size >= 4096:
+                        g[2048: 2048 + 16] = 0x7FC0                              # one whole thread tile of NaN
+            for i, g in enumerate(grads):
+                dev.tensors[i].grad.view(torch.int16).copy_(torch.from_numpy(g.view(np.int16)))
+            dev.step(step)
+            ora.step(step, grads)
+            torch.cuda.synchronize()
+            dev.check_guards()
+            for i, t in enumerate(w.tensors):
+                d = dev.tensors[i]
+                tag = f"step {step} tensor {i} [{t.rows}x{t.cols}]"
+                assert (_np(d.w) == ora.w[i]).all(), tag + ": codes"
+                assert (_scale_bits(d.scale) == _oracle_scale_bits(ora.scale[i])).all(), tag + ": scales"
+                for got, ref in ((_np(d.m), ora.m[i]),) + (((_np(d.v), ora.v[i]),) if opt == wl.ADAM else ()):
+                    nan = np.isnan(ref)
+                    assert (np.isnan(got) == nan).all(), tag + ": NaN positions"
+                    assert (got[~nan].view(np.int32) == ref[~nan].view(np.int32)).all(), tag + ": finite moments differ in their bits"
+                if step >= 2:
+                    assert np.isnan(ora.m[i]).sum() >= special.size               # the test did contaminate something
+    finally:
+        dev.destroy()
+
+
+def _digest(buf: torch.Tensor):
+    """Order-sensitive 128-bit-per-chunk digest of a byte buffer (whole multiples of 8 bytes), computed on the device
+    in chunks of 512 MB: (sum of the 64-bit words, sum of word * odd weight by position), both modulo 2^64."""
+    v = buf.view(torch.int64)
+    chunk = 1 << 26
+    weights = torch.arange(chunk, dtype=torch.int64, device=buf.device) * 2 + 1
+    out = []
+    for o in range(0, v.numel(), chunk):
+        c = v[o: o + chunk]
+        out.append((int(c.sum()), int((c * weights[: c.numel()]).sum())))
+    return out
+
+
+def _whole_set_stream_against_direct(w: wl.Workload, steps=2):
+    """Every tensor of a full-size set, not a sample: the set is stepped by the persistent streaming kernels (ticket
+    scheduler, the configuration the benchmark times) and again, from the same seeded state, by the direct-load
+    kernels (one CTA per unit, no scheduler).  All codes, scales and moments must agree bit for bit: a unit that the
+    scheduler skipped, ran twice or handed to the wrong tensor anywhere in the set shows.  (The direct-load kernels
+    are held to the oracle on the same shapes by the sampled and the ragged-shape tests.)  Where two copies of the
+    state fit the device the buffers are compared directly, otherwise through position-weighted digests."""
+    free, _ = torch.cuda.mem_get_info()
+    adam = w.optimizer == wl.ADAM
+    state = sum(w.code_bytes(t) + t.numel * (8 if adam else 4) for t in w.tensors)
+    need_one = state + 2 * w.numel
+    if free < need_one + 6 * 2 ** 30:
+        pytest.skip(f"needs {need_one / 2 ** 30:.0f} GB of device memory")
+    keep_copy = free > need_one + state + 12 * 2 ** 30
+    results = []
+    for use_stream in (1, 0):
+        eco.eco_set_option("use_stream", use_stream)
+        try:
+            dev = DeviceState(w)
+            dev.init_on_device(seed=91)
+            dev.set_grads_on_device(seed=92)
+            dev.create()
+        finally:
+            eco.eco_set_option("use_stream", 1)
+        try:
+            for step in range(1, steps + 1):
+                dev.step(step)
+            torch.cuda.synchronize()
+            eco.eco_check(dev.handle, torch.cuda.current_stream().cuda_stream)
+            dev.check_guards()
+            bufs = [b for b in (dev.w_buf, dev.s_buf, dev.m_buf, dev.v_buf) if b is not None]
+            if use_stream == 1:
+                results = [b.clone() for b in bufs] if keep_copy else [_digest(b) for b in bufs]
+            else:
+                for name, b, ref in zip(("codes", "scales", "m", "v"), bufs, results):
+                    if keep_copy:
+                        assert torch.equal(b, ref), f"{w.name}: {name} differ between the streaming and the direct-load kernels"
+                    else:
+                        got = _digest(b)
+                        bad = [k for k, (x, y) in enumerate(zip(got, ref)) if x != y]
+                        assert not bad, f"{w.name}: {name} differ in 512 MB chunks {bad[:8]}"
+        finally:
+            dev.destroy()
+            del dev
+            torch.cuda.empty_cache()
+
+
+def test_c3_whole_set_streaming_equals_direct_load():
+    _whole_set_stream_against_direct(wl.c3())
+
+
+def test_c4_whole_set_streaming_equals_direct_load():
+    _whole_set_stream_against_direct(wl.c4())
+
+
+def test_c5_whole_set_streaming_equals_direct_load():
+    _whole_set_stream_against_direct(wl.c5())
