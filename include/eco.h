@@ -288,6 +288,14 @@ eco_status eco_attach_error_buffers(eco_ctx* ctx, float* const* e, size_t n);
  */
 eco_status eco_selftest_wait(eco_ctx* ctx, int64_t limit_cycles, void* cuda_stream);
 
+/*
+ * eco_selftest_grid_wait -- the same for the one wait between CTAs that the library has: the grid barrier of the
+ * single-launch per-tensor step ("fused_tensor").  Two CTAs meet at a barrier that expects a third arrival, with
+ * a limit of limit_cycles (1..2e9); the wait must expire, record its code and let the kernel end normally.
+ * Returns ECO_ERR_TIMEOUT when the mechanism works; clears the status word again.  Call it between steps.
+ */
+eco_status eco_selftest_grid_wait(eco_ctx* ctx, int64_t limit_cycles, void* cuda_stream);
+
 /* eco_destroy -- free the context's tables and scratch (synchronizes the device). NULL is allowed. */
 eco_status eco_destroy(eco_ctx* ctx);
 
@@ -338,6 +346,12 @@ eco_status eco_dequantize(const eco_config* cfg, const void* w, const void* scal
  *                     the direct-load kernels everywhere
  *   "ctas_per_sm"     persistent grid size in CTAs per SM, 1..3; 0 (default) = as many as the kernel is built to
  *                     keep resident (3 for momentum SGD, 2 for Adam)
+ *   "fused_tensor"    per-tensor scales only: run both passes in ONE cooperative launch, wave by wave (a wave = whole
+ *                     tensors with about an L2's worth of inputs; the grid meets at a bounded barrier between the
+ *                     passes of a wave, and pass 2 finds the wave in shared memory and L2).  0 never, 1 always,
+ *                     2 (default) when the whole context is a single wave.  eco_step_begin / eco_step_end always
+ *                     use two launches (the exchange sits between them)
+ *   "wave_bytes"      input bytes of a wave (default 100 MiB; at least 1 MiB)
  * No option changes any result bit.  Errors: ECO_ERR_INVALID_ARG for an unknown name.
  */
 eco_status eco_set_option(const char* name, int64_t value);

@@ -24,13 +24,15 @@ namespace {
 thread_local std::string g_thread_error;
 
 enum LaunchKind { KIND_BLOCK_FAST = 0, KIND_BLOCK_GENERIC = 1, KIND_TENSOR = 2, KIND_ROW = 3, KIND_TENSOR_STREAM = 4,
-                  KIND_ROW_STREAM = 5 };
+                  KIND_ROW_STREAM = 5, KIND_TENSOR_WAVE = 6 };
 
 struct Launch {
     int kind;
     size_t desc_offset;   // into d_descs
     size_t unit_offset;   // into d_unit_tensor
     uint32_t n_units;
+    size_t wave_offset = 0;   // KIND_TENSOR_WAVE: into d_waves
+    uint32_t n_waves = 0;
 };
 
 // Options settable through eco_set_option before eco_create.
@@ -39,6 +41,9 @@ struct Options {
     int64_t reverse_pass2 = 1;     // per-tensor scale: walk pass 2 in the opposite order of pass 1
     int64_t use_stream = 1;        // 1: TMA-fed persistent kernels where the layout allows; 0: direct-load kernels only
     int64_t ctas_per_sm = 0;       // persistent grid = ctas_per_sm * SM count; 0: the kernel's own residency (2 or 3)
+    int64_t fused_tensor = 2;      // per-tensor scale: both passes in one cooperative launch, wave by wave: 0 = never (launch
+                                   // pair), 1 = always, 2 = when the whole context is a single wave (see eco_create)
+    int64_t wave_bytes = 100ll << 20;   // per-tensor scale, one launch: input bytes of a wave of tensors (about the L2 size)
 };
 Options g_options;
 
@@ -55,6 +60,8 @@ struct eco_ctx {
     float* d_s_old = nullptr;
     uint32_t* d_status = nullptr;
     uint32_t* d_tickets = nullptr;
+    eco::WaveDesc* d_waves = nullptr;
+    uint32_t* d_grid_counter = nullptr;
     bool pending = false;          // eco_step_begin issued, eco_step_end not yet
     std::vector<TensorDesc> h_descs;      // host copy of the descriptor table (patched by eco_attach_error_buffers)
     std::vector<size_t> desc_of_tensor;   // tensor index -> its descriptor
@@ -241,6 +248,12 @@ eco_status eco_set_option(const char* name, int64_t value) {
     if (!std::strcmp(name, "l2_group_bytes")) { g_options.l2_group_bytes = value; return ECO_OK; }
     if (!std::strcmp(name, "reverse_pass2")) { g_options.reverse_pass2 = value; return ECO_OK; }
     if (!std::strcmp(name, "use_stream")) { g_options.use_stream = value; return ECO_OK; }
+    if (!std::strcmp(name, "fused_tensor")) { g_options.fused_tensor = value; return ECO_OK; }
+    if (!std::strcmp(name, "wave_bytes")) {
+        if (value < (1 << 20)) return fail(nullptr, ECO_ERR_INVALID_ARG, "wave_bytes must be at least 1 MiB");
+        g_options.wave_bytes = value;
+        return ECO_OK;
+    }
     if (!std::strcmp(name, "ctas_per_sm")) {
         if (value < 0 || value > 3) return fail(nullptr, ECO_ERR_INVALID_ARG, "ctas_per_sm must be 0 (automatic), 1, 2 or 3");
         g_options.ctas_per_sm = value;
@@ -313,6 +326,10 @@ eco_status eco_create(eco_ctx** out, const eco_config* cfg, const eco_tensor* te
     const uint64_t rpu = static_cast<uint64_t>(eco::rows_per_unit());
     std::vector<TensorDesc> descs;
     std::vector<uint32_t> unit_tensor;
+    std::vector<eco::WaveDesc> waves;
+    int coop_attr = 0;
+    cudaDeviceGetAttribute(&coop_attr, cudaDevAttrCooperativeLaunch, device);
+    const bool cooperative = coop_attr != 0;
     auto base_desc = [&](size_t i) {
         const eco_tensor& t = tensors[i];
         TensorDesc d;
@@ -351,7 +368,7 @@ eco_status eco_create(eco_ctx** out, const eco_config* cfg, const eco_tensor* te
                 d.unit_rows = (static_cast<uint32_t>(eco::stream_unit_rows()) / d.blocks_per_row) * d.blocks_per_row;
                 nu = (d.n_blocks + d.unit_rows - 1) / d.unit_rows;
             } else {
-                d.n_blocks = (kind == KIND_TENSOR || kind == KIND_TENSOR_STREAM) ? (d.numel + 127) / 128
+                d.n_blocks = (kind == KIND_TENSOR || kind == KIND_TENSOR_STREAM || kind == KIND_TENSOR_WAVE) ? (d.numel + 127) / 128
                                                    : static_cast<uint64_t>(tensors[members[k]].rows) * d.blocks_per_row;
                 nu = (d.n_blocks + rpu - 1) / rpu;
             }
@@ -367,6 +384,10 @@ eco_status eco_create(eco_ctx** out, const eco_config* cfg, const eco_tensor* te
         return true;
     };
 
+    double context_in_bytes = 0;      // input bytes of one step over the whole context
+    for (size_t i = 0; i < n; ++i)
+        context_in_bytes += ((cfg->format == ECO_FORMAT_INT4 ? 0.5 : 1.0) + 2.0 + (adam ? 8.0 : 4.0)) *
+                            static_cast<double>(tensors[i].rows) * static_cast<double>(tensors[i].cols);
     bool ok = true;
     if (cfg->granularity == ECO_SCALE_PER_BLOCK) {
         std::vector<size_t> fast, generic;
@@ -382,6 +403,52 @@ eco_status eco_create(eco_ctx** out, const eco_config* cfg, const eco_tensor* te
         }
         ok = add_launch(KIND_ROW_STREAM, fast) && add_launch(KIND_ROW, generic);
         ctx->num_launches = static_cast<int>(ctx->launches.size());
+    } else if (use_stream && cooperative && g_options.l2_group_bytes == 0 &&
+               (g_options.fused_tensor == 1 || (g_options.fused_tensor == 2 && context_in_bytes <= static_cast<double>(g_options.wave_bytes)))) {
+        // Per-tensor scale, one cooperative launch: waves of whole tensors whose inputs are about as large as L2.  A
+        // tensor of at least half the budget is a wave of its own; smaller ones are packed in the order given.
+        // Default: only when the whole context is one wave (it then stays on the chip between the passes and the step
+        // is a single launch).  On larger sets the launch pair is faster although it moves more bytes: with two front
+        // halves the step is bound by instruction issue, and the grid barrier of every wave idles the SMs that arrive early.
+        const double in_bytes_per_elem = (cfg->format == ECO_FORMAT_INT4 ? 0.5 : 1.0) + 2.0 + (adam ? 8.0 : 4.0);
+        const double budget = static_cast<double>(g_options.wave_bytes);
+        std::vector<std::vector<size_t>> groups;
+        std::vector<size_t> small, generic;
+        double small_bytes = 0;
+        for (size_t i = 0; i < n; ++i) {
+            const uint64_t numel = static_cast<uint64_t>(tensors[i].rows) * static_cast<uint64_t>(tensors[i].cols);
+            if (numel % 128 != 0) { generic.push_back(i); continue; }
+            const double b = in_bytes_per_elem * static_cast<double>(numel);
+            if (b >= budget / 2) { groups.push_back({i}); continue; }
+            if (!small.empty() && small_bytes + b > budget) {
+                groups.push_back(small);
+                small.clear();
+                small_bytes = 0;
+            }
+            small.push_back(i);
+            small_bytes += b;
+        }
+        if (!small.empty()) groups.push_back(small);
+        std::vector<size_t> members;
+        for (const auto& g : groups) members.insert(members.end(), g.begin(), g.end());
+        ok = add_launch(KIND_TENSOR_WAVE, members);
+        if (ok && !members.empty()) {
+            Launch& L = ctx->launches.back();
+            L.wave_offset = waves.size();
+            size_t k = 0;
+            for (const auto& g : groups) {
+                eco::WaveDesc wd;
+                wd.first_unit = descs[L.desc_offset + k].first_unit;
+                const TensorDesc& last = descs[L.desc_offset + k + g.size() - 1];
+                const uint32_t last_units = static_cast<uint32_t>((last.n_blocks + rpu - 1) / rpu);
+                wd.n_units = last.first_unit + last_units - wd.first_unit;
+                waves.push_back(wd);
+                k += g.size();
+            }
+            L.n_waves = static_cast<uint32_t>(groups.size());
+        }
+        if (ok) ok = add_launch(KIND_TENSOR, generic);
+        ctx->num_launches = (members.empty() ? 0 : 1) + (generic.empty() ? 0 : 2);
     } else {
         // Per-tensor scale: pass 1 + pass 2 per group of tensors whose inputs fit the L2 budget, so
         // that pass 2 finds what pass 1 read still cached.
@@ -444,6 +511,12 @@ eco_status eco_create(eco_ctx** out, const eco_config* cfg, const eco_tensor* te
     ECO_CUDA_CTX(cudaMemset(ctx->d_status, 0, sizeof(uint32_t)));
     ECO_CUDA_CTX(cudaMalloc(&ctx->d_tickets, 2 * sizeof(uint32_t)));
     ECO_CUDA_CTX(cudaMemset(ctx->d_tickets, 0, 2 * sizeof(uint32_t)));
+    if (!waves.empty()) {
+        ECO_CUDA_CTX(cudaMalloc(&ctx->d_waves, waves.size() * sizeof(eco::WaveDesc)));
+        ECO_CUDA_CTX(cudaMemcpy(ctx->d_waves, waves.data(), waves.size() * sizeof(eco::WaveDesc), cudaMemcpyHostToDevice));
+        ECO_CUDA_CTX(cudaMalloc(&ctx->d_grid_counter, 2 * sizeof(uint32_t)));
+        ECO_CUDA_CTX(cudaMemset(ctx->d_grid_counter, 0, 2 * sizeof(uint32_t)));
+    }
     ECO_CUDA_CTX(cudaDeviceSynchronize());
 #undef ECO_CUDA_CTX
     *out = ctx;
@@ -543,6 +616,23 @@ eco_status enqueue_step(eco_ctx* ctx, const StepParams& P, void* cuda_stream, in
                                                      ctx->d_amax[parity], ctx->d_amax[parity ^ 1], ctx->d_s_old,
                                                      ctx->reverse_pass2, ctx->d_tickets, ctx->d_status, ctx->grid_cap, stream, ctx->has_error_buffers));
                 break;
+            case KIND_TENSOR_WAVE:
+                if (pass == PASS_BOTH) {
+                    ECO_CUDA(ctx, eco::launch_wave(ctx->lc, descs, units, ctx->d_waves + L.wave_offset, L.n_waves, P,
+                                                   ctx->d_amax[parity], ctx->d_amax[parity ^ 1], ctx->d_s_old,
+                                                   ctx->d_grid_counter, ctx->d_status, ctx->grid_cap, stream, ctx->has_error_buffers));
+                    break;
+                }
+                // the step cut in two for an amax exchange between ranks: the two passes as separate launches
+                if (pass != PASS_APPLY)
+                    ECO_CUDA(ctx, eco::launch_stream(ctx->lc, eco::STREAM_TENSOR_AMAX, descs, units, L.n_units, P,
+                                                     ctx->d_amax[parity], nullptr, ctx->d_s_old, false, ctx->d_tickets,
+                                                     ctx->d_status, ctx->grid_cap, stream));
+                if (pass != PASS_AMAX)
+                    ECO_CUDA(ctx, eco::launch_stream(ctx->lc, eco::STREAM_TENSOR_APPLY, descs, units, L.n_units, P,
+                                                     ctx->d_amax[parity], ctx->d_amax[parity ^ 1], ctx->d_s_old,
+                                                     ctx->reverse_pass2, ctx->d_tickets, ctx->d_status, ctx->grid_cap, stream, ctx->has_error_buffers));
+                break;
             case KIND_ROW:
                 ECO_CUDA(ctx, eco::launch_row(ctx->lc, descs, units, L.n_units, P, stream));
                 break;
@@ -574,7 +664,8 @@ eco_status eco_check(eco_ctx* ctx, void* cuda_stream) {
     ECO_CUDA(ctx, cudaMemcpy(&code, ctx->d_status, sizeof code, cudaMemcpyDeviceToHost));
     if (code != 0)
         return fail(ctx, ECO_ERR_TIMEOUT, "a bounded wait inside a kernel expired (code %u: 1 = producer waiting for a free "
-                    "stage, 2 = producer draining its copies, 3 = consumer waiting for data, 4/5 = per-row exchange, 7 = self-test)", code);
+                    "stage, 2 = producer draining its copies, 3 = consumer waiting for data, 4/5 = per-row exchange, 6 = grid barrier of the "
+                    "single-launch per-tensor step, 7 = self-test, 8 = consumer warps meeting)", code);
     return ECO_OK;
 }
 
@@ -605,6 +696,21 @@ eco_status eco_selftest_wait(eco_ctx* ctx, int64_t limit_cycles, void* cuda_stre
     return st;
 }
 
+eco_status eco_selftest_grid_wait(eco_ctx* ctx, int64_t limit_cycles, void* cuda_stream) {
+    if (!ctx) return fail(nullptr, ECO_ERR_INVALID_ARG, "ctx is NULL");
+    if (limit_cycles < 1 || limit_cycles > 2000000000LL)
+        return fail(ctx, ECO_ERR_INVALID_ARG, "limit_cycles must be in 1..2e9 (got %lld)", static_cast<long long>(limit_cycles));
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    // the self-test's arrival counter: the context's ticket words, which are zero between steps (and zeroed again below)
+    ECO_CUDA(ctx, cudaMemsetAsync(ctx->d_tickets, 0, 2 * sizeof(uint32_t), stream));
+    ECO_CUDA(ctx, eco::launch_grid_wait_selftest(ctx->d_tickets, ctx->d_status, limit_cycles, stream));
+    const eco_status st = eco_check(ctx, cuda_stream);
+    ECO_CUDA(ctx, cudaMemsetAsync(ctx->d_status, 0, sizeof(uint32_t), stream));
+    ECO_CUDA(ctx, cudaMemsetAsync(ctx->d_tickets, 0, 2 * sizeof(uint32_t), stream));
+    ECO_CUDA(ctx, cudaStreamSynchronize(stream));
+    return st;
+}
+
 eco_status eco_destroy(eco_ctx* ctx) {
     if (!ctx) return ECO_OK;
     cudaSetDevice(ctx->device);
@@ -616,6 +722,8 @@ eco_status eco_destroy(eco_ctx* ctx) {
     cudaFree(ctx->d_s_old);
     cudaFree(ctx->d_status);
     cudaFree(ctx->d_tickets);
+    cudaFree(ctx->d_waves);
+    cudaFree(ctx->d_grid_counter);
     delete ctx;
     return ECO_OK;
 }

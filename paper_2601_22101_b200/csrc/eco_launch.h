@@ -38,8 +38,24 @@ cudaError_t launch_stream(const LaunchConfig& c, int mode, const TensorDesc* des
                           bool reverse, uint32_t* tickets, uint32_t* status, int grid_cap, cudaStream_t stream,
                           bool with_errors = false);
 
+// A wave of the single-launch per-tensor step: the units [first_unit, first_unit + n_units) of the launch's unit table,
+// made of whole tensors.
+struct WaveDesc {
+    uint32_t first_unit, n_units;
+};
+
+// Per-tensor scales in one cooperative launch (see eco_wave_kernel): both passes of every wave, a grid barrier in
+// between.  `grid_counter`: two device words, zero before the first launch, rewound by the kernel itself.  The grid is
+// the number of CTAs the device can hold at once (or grid_cap, if that is smaller).
+cudaError_t launch_wave(const LaunchConfig& c, const TensorDesc* descs, const uint32_t* unit_tensor, const WaveDesc* waves,
+                        uint32_t n_waves, const StepParams& P, uint32_t* amax, uint32_t* amax_next, float* s_old,
+                        uint32_t* grid_counter, uint32_t* status, int grid_cap, cudaStream_t stream, bool with_errors);
+
 // One warp waits, for at most limit_cycles, on a barrier nothing arrives on; then writes code 7 to *status.
 cudaError_t launch_wait_selftest(uint32_t* status, long long limit_cycles, cudaStream_t stream);
+// Two CTAs wait, for at most limit_cycles, at a grid barrier that expects a third; then code 6 is written to *status.
+// `counter`: a device word, zero before the launch (left non-zero).
+cudaError_t launch_grid_wait_selftest(uint32_t* counter, uint32_t* status, long long limit_cycles, cudaStream_t stream);
 
 cudaError_t launch_block128(const LaunchConfig& c, const TensorDesc* descs, const uint32_t* unit_tensor,
                             uint32_t n_units, bool generic, const StepParams& P, cudaStream_t stream);

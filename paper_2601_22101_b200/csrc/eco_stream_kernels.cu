@@ -44,10 +44,12 @@ struct StageHeader {
     uint32_t seg_per_row; // per-row mode: 128-element rows per matrix row (R)
     uint32_t div_magic;   // per-row mode: floor(65536 / R) + 1, so that (x * div_magic) >> 16 == x / R for x < 2048
     uint32_t n_mrows;     // per-row mode: matrix rows in the unit
-    uint32_t pad_;
+    uint32_t pass;        // wave kernel: what this publication is (WAVE_*)
     uint64_t mrow0;       // per-row mode: first matrix row of the unit
     uint64_t index_base;  // element index of the tensor's first element inside the full (unsharded) tensor
     float* e;             // optional error buffer of the tensor (NULL: none)
+    uint32_t barrier_target;   // wave kernel: non-zero = wait until the grid counter reaches this before going on
+    uint32_t first_of_tensor;  // wave kernel: this unit is the first of its tensor (its consumers store the new scale)
 };
 static_assert(sizeof(StageHeader) <= 128, "header must fit its slot");
 
@@ -111,6 +113,27 @@ __device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_
                  ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
 }
 
+// The same with an L2 eviction-priority hint (a policy made by createpolicy) for this copy's lines.
+__device__ __forceinline__ void bulk_load_hint(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar, uint64_t policy) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;"
+                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar), "l"(policy) : "memory");
+}
+__device__ __forceinline__ uint64_t policy_evict_first() {
+    uint64_t p;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
+    return p;
+}
+// 16- and 4/2-byte stores whose lines L2 may drop first (results that are not read again within the step).
+__device__ __forceinline__ void store_f4_first(float* p, float a, float b, float c, float d, uint64_t policy) {
+    asm volatile("st.global.L2::cache_hint.v4.f32 [%0], {%1, %2, %3, %4}, %5;" ::"l"(p), "f"(a), "f"(b), "f"(c), "f"(d), "l"(policy) : "memory");
+}
+__device__ __forceinline__ void store_u32_first(void* p, uint32_t v, uint64_t policy) {
+    asm volatile("st.global.L2::cache_hint.u32 [%0], %1, %2;" ::"l"(p), "r"(v), "l"(policy) : "memory");
+}
+__device__ __forceinline__ void store_u16_first(void* p, uint32_t v, uint64_t policy) {
+    asm volatile("st.global.L2::cache_hint.u16 [%0], %1, %2;" ::"l"(p), "h"(static_cast<uint16_t>(v)), "l"(policy) : "memory");
+}
+
 // max |x| over the 32 lanes in one instruction (sm_100a warp reduction on binary32; NaN operands are
 // ignored, as by fmaxf).  Every lane receives the result.  The final maximum with zero makes a warp whose
 // operands are ALL NaN return 0 (a block of nothing but NaN has no maximum: it takes the scale of an all-zero block).
@@ -126,12 +149,17 @@ __device__ __forceinline__ uint32_t units_of(const TensorDesc& T) {
 
 // One unit (up to 32 rows of 128 elements) by the 8 consumer warps: warp w owns rows 4w..4w+3, lane l
 // elements 4l..4l+3 of each.  FULL: all 32 rows are present (every unit but the last of a tensor).
-template <int FMT, int OPT, int RND, int MODE, bool FULL, bool ERR, int NS = 4>
+// TS: the scales of the per-tensor modes (old scale for the dequantization; new scale and its inverse for pass 2).
+struct TensorScales { float s_old, s_new, inv_new; };
+// HINT: stores carry an evict-first hint (`store_policy`); false = plain stores.
+template <int FMT, int OPT, int RND, int MODE, bool FULL, bool ERR, int NS = 4, bool HINT = false>
 __device__ __forceinline__ bool consume_unit(const StepParams& P, const int scale_kind, const uint8_t* st,
                                              const StageHeader* h, const uint32_t empty_bar, const int warp,
                                              const int lane, uint32_t* scratch_amax, uint32_t& cur_slot,
                                              float& run_max, float* xchg, const uint32_t row_bars,
-                                             const uint32_t row_parity, uint32_t* status) {
+                                             const uint32_t row_parity, uint32_t* status,
+                                             const TensorScales ts = TensorScales{1.0f, 1.0f, 1.0f},
+                                             const uint64_t store_policy = 0) {
     using SL = StageLayout<FMT, OPT>;
     // Row (of 128 elements) behind slot k of this warp.  Per-row mode deals the rows round-robin (warp, warp + 8, ...)
     // so that a unit of fewer than 32 rows leaves every warp with 3 or 4 rows instead of some with none; NS is the
@@ -172,7 +200,7 @@ __device__ __forceinline__ bool consume_unit(const StepParams& P, const int scal
                 if (MODE == MODE_BLOCK) s_old = reinterpret_cast<const float*>(st + SL::kScales)[row];
                 else if (MODE == MODE_BLOCK32) s_old = reinterpret_cast<const float*>(st + SL::kScales)[row * 4 + (lane >> 3)];
                 else if (MODE == MODE_ROW) s_old = reinterpret_cast<const float*>(st + SL::kScales)[(row * h->div_magic) >> 16];
-                else s_old = h->s_old;
+                else s_old = ts.s_old;
             }
             float val[4];
             unpack4<FMT>(codes, val);
@@ -188,8 +216,10 @@ __device__ __forceinline__ bool consume_unit(const StepParams& P, const int scal
             const bool valid = FULL || r + k * kRowStep < nrows;
             amax[k] = 0.0f;
             if (valid) amax[k] = fmaxf(fmaxf(fabsf(L[k].tht[0]), fabsf(L[k].tht[1])), fmaxf(fabsf(L[k].tht[2]), fabsf(L[k].tht[3])));
-            if (OPT == OPT_ADAM && MODE != MODE_TENSOR_AMAX && valid)
-                *reinterpret_cast<float4*>(vp + i_first + k * (kRowStep * 128)) = make_float4(vt[k][0], vt[k][1], vt[k][2], vt[k][3]);
+            if (OPT == OPT_ADAM && MODE != MODE_TENSOR_AMAX && valid) {
+                if (HINT) store_f4_first(vp + i_first + k * (kRowStep * 128), vt[k][0], vt[k][1], vt[k][2], vt[k][3], store_policy);
+                else *reinterpret_cast<float4*>(vp + i_first + k * (kRowStep * 128)) = make_float4(vt[k][0], vt[k][1], vt[k][2], vt[k][3]);
+            }
         }
     }
     // everything needed later is read before the stage is handed back
@@ -198,7 +228,7 @@ __device__ __forceinline__ bool consume_unit(const StepParams& P, const int scal
     void* const sp = h->scale;
     const uint64_t row0 = h->row0;
     const uint32_t tensor_id = h->tensor_id, slot = h->slot;
-    const float s_new = h->s_new, inv_new = h->inv_new;
+    const float s_new = ts.s_new, inv_new = ts.inv_new;
     const uint32_t seg_per_row = h->seg_per_row, div_magic = h->div_magic, n_mrows = h->n_mrows;
     const uint64_t mrow0 = h->mrow0, index_base = h->index_base;
     float* const ep = h->e;
@@ -319,10 +349,17 @@ __device__ __forceinline__ bool consume_unit(const StepParams& P, const int scal
         // float kernels with f32 / bf16 scales take the two-operation form without asking
         constexpr int kExact = MODE == MODE_BLOCK32 ? 1 : (FMT == FMT_INT4 ? -1 : 0);
         const uint32_t codes = back4<FMT, OPT, RND, ERR, kExact>(P, word, s_k[k], inv_k[k], L[k], mh, e_prev, e_out);
-        if (FMT != FMT_INT4) *reinterpret_cast<uint32_t*>(wp + i0) = codes;
-        else *reinterpret_cast<uint16_t*>(wp + (i0 >> 1)) = static_cast<uint16_t>(codes);
-        *reinterpret_cast<float4*>(mp + i0) = make_float4(mh[0], mh[1], mh[2], mh[3]);
-        if (ERR) *reinterpret_cast<float4*>(ep + i0) = make_float4(e_out[0], e_out[1], e_out[2], e_out[3]);
+        if (HINT) {
+            if (FMT != FMT_INT4) store_u32_first(wp + i0, codes, store_policy);
+            else store_u16_first(wp + (i0 >> 1), codes, store_policy);
+            store_f4_first(mp + i0, mh[0], mh[1], mh[2], mh[3], store_policy);
+            if (ERR) store_f4_first(ep + i0, e_out[0], e_out[1], e_out[2], e_out[3], store_policy);
+        } else {
+            if (FMT != FMT_INT4) *reinterpret_cast<uint32_t*>(wp + i0) = codes;
+            else *reinterpret_cast<uint16_t*>(wp + (i0 >> 1)) = static_cast<uint16_t>(codes);
+            *reinterpret_cast<float4*>(mp + i0) = make_float4(mh[0], mh[1], mh[2], mh[3]);
+            if (ERR) *reinterpret_cast<float4*>(ep + i0) = make_float4(e_out[0], e_out[1], e_out[2], e_out[3]);
+        }
     }
     return true;
 }
@@ -422,7 +459,7 @@ eco_stream_kernel(const TensorDesc* __restrict__ descs, const uint32_t* __restri
                 h.row0 = row0; h.nrows = nrows; h.tensor_id = T.tensor_id; h.slot = T.slot;
                 h.s_old = 1.0f; h.s_new = 1.0f; h.inv_new = 1.0f;
                 h.seg_per_row = T.blocks_per_row; h.div_magic = 65536u / T.blocks_per_row + 1u;
-                h.n_mrows = n_mrows; h.pad_ = 0u; h.mrow0 = mrow0; h.index_base = T.index_base; h.e = T.e;
+                h.n_mrows = n_mrows; h.pass = 0u; h.barrier_target = 0u; h.first_of_tensor = 0u; h.mrow0 = mrow0; h.index_base = T.index_base; h.e = T.e;
                 if (MODE == MODE_TENSOR_AMAX) {
                     h.s_old = load_scale(T.scale, 0, scale_kind);
                     if (local == 0) scratch_s_old[T.slot] = h.s_old;
@@ -504,16 +541,360 @@ eco_stream_kernel(const TensorDesc* __restrict__ descs, const uint32_t* __restri
                                                                       run_max, xchg, row_bars, it & 1u, status);
         } else if (nrows == kUnitRows)   // (discarded statement of the if constexpr above for the per-row mode)
             ok = consume_unit<FMT, OPT, RND, MODE, true, ERR>(P, scale_kind, st, h, empty, warp, lane, scratch_amax, cur_slot,
-                                                              run_max, xchg, row_bars, it & 1u, status);
+                                                              run_max, xchg, row_bars, it & 1u, status,
+                                                              TensorScales{h->s_old, h->s_new, h->inv_new});
         else
             ok = consume_unit<FMT, OPT, RND, MODE, false, ERR>(P, scale_kind, st, h, empty, warp, lane, scratch_amax, cur_slot,
-                                                               run_max, xchg, row_bars, it & 1u, status);
+                                                               run_max, xchg, row_bars, it & 1u, status,
+                                                               TensorScales{h->s_old, h->s_new, h->inv_new});
         if (!ok) return;
     }
     if (MODE == MODE_TENSOR_AMAX && cur_slot != 0xFFFFFFFFu) {
         const float z = warp_amax(run_max);
         if (lane == 0) atomicMax(scratch_amax + cur_slot, __float_as_uint(z));
     }
+}
+
+// ---------------------------------------------------------------------------
+// Per-tensor scale in ONE cooperative launch: the parameter set is cut into waves of whole tensors whose inputs
+// are about as large as L2 (a tensor larger than that is a wave of its own).  Wave by wave, every CTA streams its
+// share of the wave's units once for max |theta~| (pass 1), the grid meets at a barrier, and the CTA goes over the
+// same units again (pass 2) with the now complete maxima: first the units still sitting in its shared-memory stages
+// (no load at all), then the others newest first, which the L2 still holds for the most part.  A tensor that fits
+// the chip is therefore read from HBM once (20 B/param for FP8 + Adam) instead of twice (31).
+//
+// CTA c of G owns units c, c + G, ... of every wave: the same SM touches the same addresses in both passes.
+// The producer warp publishes a sequence of stages (round-robin over the ring); a publication is one of
+//   WAVE_AMAX    a freshly loaded unit, pass 1
+//   WAVE_APPLY   a unit for pass 2: freshly loaded, or -- `resident` -- the stage as pass 1 left it (nothing is copied)
+//   WAVE_NOOP    nothing (keeps the ring position in step when a CTA has fewer units in a wave than stages)
+//   WAVE_END     end of the kernel
+// The first pass-2 publication of a wave (a no-op if the CTA has no unit there) carries the barrier: before they
+// process it, the consumer warps post their maxima, one thread arrives on the grid counter and waits, bounded, until
+// every CTA has arrived.  The producer never waits for the grid: it goes on issuing the copies of pass 2 while the
+// consumers stand at the barrier, so the memory system stays busy across it.  Launched cooperatively, so that all
+// CTAs are resident and the barrier can complete.
+// L2 hints (measured with a probe of this access pattern): the units that will stay in shared memory, the re-loads of
+// pass 2 and all stores are marked evict-first, which leaves the L2 to the lines pass 2 still needs.
+// ---------------------------------------------------------------------------
+enum : uint32_t { WAVE_AMAX = 1, WAVE_APPLY = 2, WAVE_NOOP = 3, WAVE_END = 4 };
+
+#ifdef ECO_WAVE_TRACE
+// Development aid, not compiled into the library: nanosecond timestamps of every CTA at four points of every wave
+// (first unit of pass 1 in hand, arrival at the barrier, release from it, first unit of the next wave in hand).
+constexpr uint32_t kTraceWaves = 128, kTraceCtas = 512;
+__device__ unsigned long long g_wave_trace[kTraceCtas * kTraceWaves * 4];
+__device__ __forceinline__ void wave_trace(uint32_t wave, int point) {
+    if (threadIdx.x == 0 && wave < kTraceWaves && blockIdx.x < kTraceCtas) {
+        unsigned long long t;
+        asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+        g_wave_trace[(blockIdx.x * kTraceWaves + wave) * 4 + point] = t;
+    }
+}
+#define ECO_TRACE(wave, point) wave_trace(wave, point)
+#else
+#define ECO_TRACE(wave, point)
+#endif
+constexpr uint32_t kGridBarrierTimeout = 6u;       // status code
+
+// Meeting point of the 8 consumer warps of a CTA on an mbarrier of its own (count 8), bounded like every other wait.
+__device__ __forceinline__ bool consumers_sync(uint32_t bar, uint32_t& phase, int lane, uint32_t* status) {
+    __syncwarp();
+    if (lane == 0) mbar_arrive(bar);
+    const bool ok = mbar_wait(bar, phase & 1u, status, 8u);
+    ++phase;
+    return ok;
+}
+
+// Bounded grid barrier for the consumer warps of a CTA: they meet, one thread arrives on the grid counter and waits
+// until every CTA has, they meet again.  Returns false when a wait ran out (the code is in *status).
+__device__ __forceinline__ bool wave_grid_barrier(uint32_t* counter, uint32_t target, uint32_t* status, uint32_t* abort_flag,
+                                                  uint32_t bar, uint32_t& phase, int lane,
+                                                  long long limit_cycles = kWaitLimitCycles) {
+    if (!consumers_sync(bar, phase, lane, status)) return false;         // every warp has posted its maxima
+    if (threadIdx.x == 0) {
+        __threadfence();
+        atomicAdd(counter, 1u);
+        const long long t0 = clock64();
+        uint32_t seen;
+        for (;;) {
+            asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(seen) : "l"(counter) : "memory");
+            if (seen >= target) break;
+            if (clock64() - t0 > limit_cycles) {
+                atomicExch(status, kGridBarrierTimeout);
+                *reinterpret_cast<volatile uint32_t*>(abort_flag) = 1u;
+                break;
+            }
+        }
+        __threadfence();
+    }
+    if (!consumers_sync(bar, phase, lane, status)) return false;
+    return *reinterpret_cast<volatile uint32_t*>(abort_flag) == 0u;
+}
+
+template <int FMT, int OPT, int RND, bool ERR>
+__global__ void __launch_bounds__(kStreamThreads, stream_ctas_per_sm<OPT, ERR>())
+eco_wave_kernel(const TensorDesc* __restrict__ descs, const uint32_t* __restrict__ unit_tensor,
+                const WaveDesc* __restrict__ waves, const uint32_t n_waves, const StepParams P, const int scale_kind,
+                uint32_t* __restrict__ scratch_amax, uint32_t* __restrict__ scratch_amax_next,
+                float* __restrict__ scratch_s_old, uint32_t* __restrict__ grid_counter, uint32_t* __restrict__ status) {
+    using SL = StageLayout<FMT, OPT>;
+    constexpr int S = SL::kStages;
+    extern __shared__ __align__(128) uint8_t smem[];
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem);
+    const uint32_t full0 = smem_addr(bars), empty0 = smem_addr(bars + S);
+    uint8_t* stage0 = smem + SL::kBarriers;
+    uint32_t* abort_flag = reinterpret_cast<uint32_t*>(smem + SL::kExchange);
+    const uint32_t sync_bar = smem_addr(smem + SL::kRowBars);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t G = gridDim.x, cta = blockIdx.x;
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < S; ++s) {
+            mbar_init(full0 + 8 * s, 2);
+            mbar_init(empty0 + 8 * s, kConsumerWarps);
+        }
+        mbar_init(sync_bar, kConsumerWarps);
+        *abort_flag = 0u;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+
+    if (warp == kConsumerWarps) {
+        // ------------------------------ producer ------------------------------
+        const uint64_t evict_first = policy_evict_first();
+        uint32_t it = 0;                         // publications so far; the next one goes to stage it % S
+        uint32_t stage_unit[S];                  // unit (index inside the wave's share) a stage holds from pass 1, or none
+        bool ok = true;
+        // Publishes one stage.  load: copy the unit's inputs in; otherwise the stage keeps what it holds.
+        uint32_t cur_ti = 0xFFFFFFFFu;           // tensor whose descriptor is in T
+        TensorDesc T;
+        float cur_s_old = 1.0f;
+        auto publish = [&](uint32_t pass, uint32_t unit, bool load, bool hint, uint32_t barrier_target) -> bool {
+            const uint32_t s = it % S, ph = (it / S) & 1;
+            if (load) {
+                // the descriptor is fetched BEFORE the wait for the stage, so that its latency hides behind that wait
+                const uint32_t ti = __ldg(unit_tensor + unit);
+                if (ti != cur_ti) {
+                    T = descs[ti];
+                    cur_ti = ti;
+                    // (read in pass 1, where the tensor's old scale is still in place; a descriptor first met in pass 2
+                    // reads the new one, which nothing uses)
+                    cur_s_old = load_scale(T.scale, 0, scale_kind);
+                }
+            }
+            if (!mbar_wait(empty0 + 8 * s, ph ^ 1, status, 1u)) return false;
+            uint8_t* st = stage0 + static_cast<size_t>(s) * SL::kBytes;
+            const uint32_t full = full0 + 8 * s;
+            if (pass == WAVE_NOOP || pass == WAVE_END) {
+                if (lane == 0) {
+                    StageHeader* h = reinterpret_cast<StageHeader*>(st + SL::kHeader);
+                    h->pass = pass;
+                    h->barrier_target = barrier_target;
+                    h->nrows = 0u;
+                    mbar_arrive_expect_tx(full, 0u);
+                }
+            } else if (!load) {
+                if (lane == 0) {                 // the stage as pass 1 left it: only the header changes
+                    StageHeader* h = reinterpret_cast<StageHeader*>(st + SL::kHeader);
+                    h->pass = pass;
+                    h->barrier_target = barrier_target;
+                    mbar_arrive_expect_tx(full, 0u);
+                }
+            } else {
+                const uint32_t local = unit - T.first_unit;
+                const uint64_t row0 = static_cast<uint64_t>(local) * kUnitRows;
+                const uint64_t left = T.n_blocks - row0;
+                const uint32_t nrows = left < kUnitRows ? static_cast<uint32_t>(left) : static_cast<uint32_t>(kUnitRows);
+                if (lane == 0) {
+                    const uint32_t cb = nrows * SL::kCodeRow, gb = nrows * 256u, mb = nrows * 512u;
+                    mbar_arrive_expect_tx(full, cb + gb + mb + (OPT == OPT_ADAM ? mb : 0u));
+                    if (hint) {
+                        bulk_load_hint(smem_addr(st + SL::kCodes), T.w + row0 * SL::kCodeRow, cb, full, evict_first);
+                        bulk_load_hint(smem_addr(st + SL::kGrad), T.grad + row0 * 128, gb, full, evict_first);
+                        bulk_load_hint(smem_addr(st + SL::kM), T.m + row0 * 128, mb, full, evict_first);
+                        if (OPT == OPT_ADAM) bulk_load_hint(smem_addr(st + SL::kV), T.v + row0 * 128, mb, full, evict_first);
+                    } else {
+                        bulk_load(smem_addr(st + SL::kCodes), T.w + row0 * SL::kCodeRow, cb, full);
+                        bulk_load(smem_addr(st + SL::kGrad), T.grad + row0 * 128, gb, full);
+                        bulk_load(smem_addr(st + SL::kM), T.m + row0 * 128, mb, full);
+                        if (OPT == OPT_ADAM) bulk_load(smem_addr(st + SL::kV), T.v + row0 * 128, mb, full);
+                    }
+                    StageHeader h;
+                    h.w = T.w; h.scale = T.scale; h.m = T.m; h.v = T.v;
+                    h.row0 = row0; h.nrows = nrows; h.tensor_id = T.tensor_id; h.slot = T.slot;
+                    h.s_old = 1.0f; h.s_new = 1.0f; h.inv_new = 1.0f;
+                    h.seg_per_row = 1u; h.div_magic = 0u; h.n_mrows = 0u; h.pass = pass; h.mrow0 = 0u;
+                    h.index_base = T.index_base; h.e = T.e;
+                    h.barrier_target = barrier_target; h.first_of_tensor = local == 0u ? 1u : 0u;
+                    if (pass == WAVE_AMAX) {
+                        // the old scale: nobody stores this tensor's new one before the wave's barrier
+                        h.s_old = cur_s_old;
+                        if (local == 0) scratch_s_old[T.slot] = cur_s_old;
+                    }
+                    *reinterpret_cast<StageHeader*>(st + SL::kHeader) = h;
+                }
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(full);
+            ++it;
+            return true;
+        };
+        for (uint32_t w = 0; w < n_waves && ok; ++w) {
+            const uint32_t first = waves[w].first_unit, n = waves[w].n_units;
+            const uint32_t mine = n > cta ? (n - cta + G - 1) / G : 0u;          // units first + cta + j G, j < mine
+#pragma unroll
+            for (int s = 0; s < S; ++s) stage_unit[s] = 0xFFFFFFFFu;
+            // pass 1; the units that end it in the stages are not needed from L2 again
+            for (uint32_t j = 0; j < mine && ok; ++j) {
+                stage_unit[it % S] = j;
+                ok = publish(WAVE_AMAX, first + cta + j * G, true, j + S >= mine, 0u);
+            }
+            if (!ok) break;
+            // pass 2: one round over the ring for what it still holds (at least one publication: it carries the barrier)
+            const uint32_t target = (w + 1u) * G;
+            uint32_t resident = mine < static_cast<uint32_t>(S) ? mine : static_cast<uint32_t>(S), k = 0;
+            do {
+                const uint32_t u = stage_unit[it % S];
+                const uint32_t bt = k == 0 ? target : 0u;
+                if (u != 0xFFFFFFFFu) {
+                    stage_unit[it % S] = 0xFFFFFFFFu;
+                    --resident;
+                    ok = publish(WAVE_APPLY, first + cta + u * G, false, false, bt);
+                } else {
+                    ok = publish(WAVE_NOOP, 0u, false, false, bt);
+                }
+                ++k;
+            } while (resident > 0 && ok);
+            // the rest of pass 2, newest first
+            if (mine > static_cast<uint32_t>(S))
+                for (uint32_t j = mine - S; j-- > 0 && ok;)
+                    ok = publish(WAVE_APPLY, first + cta + j * G, true, true, 0u);
+        }
+        if (ok) ok = publish(WAVE_END, 0u, false, false, 0u);
+        if (!ok) {
+            const uint32_t pending = it < static_cast<uint32_t>(S) ? it : static_cast<uint32_t>(S);
+            for (uint32_t k = 0; k < pending; ++k) {
+                const uint32_t j = it - 1 - k;
+                mbar_wait(full0 + 8 * (j % S), (j / S) & 1, status, 2u);
+            }
+        }
+        return;
+    }
+
+    // -------------------------------- consumers --------------------------------
+    const uint64_t evict_first = policy_evict_first();
+    uint32_t cur_slot = 0xFFFFFFFFu;
+    float run_max = 0.0f;
+    uint32_t sync_phase = 0u;
+#ifdef ECO_WAVE_TRACE
+    uint32_t trace_wave = 0u;
+    bool trace_open = false;
+#endif
+    uint32_t scale_slot = 0xFFFFFFFFu;            // tensor whose scales are in ts
+    TensorScales ts{1.0f, 1.0f, 1.0f};
+    for (uint32_t it = 0;; ++it) {
+        const uint32_t s = it % S, ph = (it / S) & 1;
+        if (!mbar_wait(full0 + 8 * s, ph, status, 3u)) return;
+        const uint8_t* st = stage0 + static_cast<size_t>(s) * SL::kBytes;
+        const StageHeader* h = reinterpret_cast<const StageHeader*>(st + SL::kHeader);
+        const uint32_t empty = empty0 + 8 * s;
+        const uint32_t pass = h->pass, nrows = h->nrows, target = h->barrier_target;
+        if (pass == WAVE_END) break;
+#ifdef ECO_WAVE_TRACE
+        if (pass == WAVE_AMAX && !trace_open) { ECO_TRACE(trace_wave, 0); trace_open = true; }
+        if (target != 0u) ECO_TRACE(trace_wave, 1);
+#endif
+        if (target != 0u) {
+            // end of this CTA's pass 1 of the wave: post the running maximum, then meet the other CTAs
+            if (cur_slot != 0xFFFFFFFFu) {
+                const float z = warp_amax(run_max);
+                if (lane == 0) atomicMax(scratch_amax + cur_slot, __float_as_uint(z));
+                cur_slot = 0xFFFFFFFFu;
+                run_max = 0.0f;
+            }
+            scale_slot = 0xFFFFFFFFu;
+            if (!wave_grid_barrier(grid_counter, target, status, abort_flag, sync_bar, sync_phase, lane)) return;
+#ifdef ECO_WAVE_TRACE
+            ECO_TRACE(trace_wave, 2);
+            ++trace_wave;
+            trace_open = false;
+#endif
+        }
+        if (pass == WAVE_NOOP) {
+            __syncwarp();
+            if (lane == 0) mbar_arrive(empty);
+            continue;
+        }
+        bool ok;
+        if (pass == WAVE_AMAX) {
+            const TensorScales t1{h->s_old, 1.0f, 1.0f};
+            if (nrows == kUnitRows)
+                ok = consume_unit<FMT, OPT, RND, MODE_TENSOR_AMAX, true, false>(P, scale_kind, st, h, empty, warp, lane, scratch_amax,
+                                                                                cur_slot, run_max, nullptr, 0u, 0u, status, t1);
+            else
+                ok = consume_unit<FMT, OPT, RND, MODE_TENSOR_AMAX, false, false>(P, scale_kind, st, h, empty, warp, lane, scratch_amax,
+                                                                                 cur_slot, run_max, nullptr, 0u, 0u, status, t1);
+        } else {
+            const uint32_t slot = h->slot;
+            if (slot != scale_slot) {
+                // the tensor's maximum is complete (barrier passed); its old scale was saved in pass 1 by the owner
+                // of its first unit.  Both were written by other SMs: read past the L1.
+                scale_slot = slot;
+                uint32_t bits;
+                ts.s_old = __ldcg(scratch_s_old + slot);
+                make_scale_div<FMT>(__uint_as_float(__ldcg(scratch_amax + slot)), scale_kind == SCALE_KIND_BF16, ts.s_new, ts.inv_new, bits);
+                if (h->first_of_tensor && warp == 0 && lane == 0) {
+                    store_scale(h->scale, 0, scale_kind, ts.s_new, bits);
+                    scratch_amax_next[slot] = 0u;
+                }
+            } else if (h->first_of_tensor && warp == 0 && lane == 0) {
+                uint32_t bits;
+                float s_new, inv_new;
+                make_scale_div<FMT>(__uint_as_float(__ldcg(scratch_amax + slot)), scale_kind == SCALE_KIND_BF16, s_new, inv_new, bits);
+                store_scale(h->scale, 0, scale_kind, s_new, bits);
+                scratch_amax_next[slot] = 0u;
+            }
+            if (nrows == kUnitRows)
+                ok = consume_unit<FMT, OPT, RND, MODE_TENSOR_APPLY, true, ERR, 4, true>(P, scale_kind, st, h, empty, warp, lane, scratch_amax,
+                                                                                       cur_slot, run_max, nullptr, 0u, 0u, status, ts, evict_first);
+            else
+                ok = consume_unit<FMT, OPT, RND, MODE_TENSOR_APPLY, false, ERR, 4, true>(P, scale_kind, st, h, empty, warp, lane, scratch_amax,
+                                                                                        cur_slot, run_max, nullptr, 0u, 0u, status, ts, evict_first);
+        }
+        if (!ok) return;
+    }
+    // the last CTA out rewinds the grid counter for the next launch (every CTA has passed every barrier by then)
+    if (!consumers_sync(sync_bar, sync_phase, lane, status)) return;
+    if (threadIdx.x == 0 && atomicAdd(grid_counter + 1, 1u) == G - 1) {
+        grid_counter[0] = 0u;
+        grid_counter[1] = 0u;
+    }
+}
+
+template <int FMT, int OPT, int RND, bool ERR>
+static cudaError_t launch_wave_one(const TensorDesc* descs, const uint32_t* unit_tensor, const WaveDesc* waves, uint32_t n_waves,
+                                   const StepParams& P, int scale_kind, uint32_t* amax, uint32_t* amax_next, float* s_old,
+                                   uint32_t* grid_counter, uint32_t* status, int grid_cap, int sm_count, cudaStream_t stream) {
+    using SL = StageLayout<FMT, OPT>;
+    static int resident = -1;                     // CTAs of this instantiation that fit one SM
+    auto kernel = eco_wave_kernel<FMT, OPT, RND, ERR>;
+    if (resident < 0) {
+        cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SL::kSmem);
+        if (e != cudaSuccess) return e;
+        int n = 0;
+        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, kernel, kStreamThreads, SL::kSmem);
+        if (e != cudaSuccess) return e;
+        if (n < 1) return cudaErrorLaunchOutOfResources;
+        resident = n < stream_ctas_per_sm<OPT, ERR>() ? n : stream_ctas_per_sm<OPT, ERR>();
+    }
+    // every CTA must be resident for the grid barrier: never more than the SMs can hold at once
+    int grid = resident * sm_count;
+    if (grid_cap > 0 && grid_cap < grid) grid = grid_cap;
+    StepParams Pc = P;
+    int sk = scale_kind;
+    void* args[] = {&descs, &unit_tensor, &waves, &n_waves, &Pc, &sk, &amax, &amax_next, &s_old, &grid_counter, &status};
+    return cudaLaunchCooperativeKernel(reinterpret_cast<void*>(kernel), dim3(grid), dim3(kStreamThreads), args, SL::kSmem, stream);
 }
 
 // ---------------------------------------------------------------------------
@@ -578,6 +959,26 @@ cudaError_t launch_stream(const LaunchConfig& c, int mode, const TensorDesc* des
     return cudaErrorInvalidValue;
 }
 
+#ifdef ECO_WAVE_TRACE
+extern "C" int eco_debug_read_wave_trace(void* host, size_t bytes) {
+    return static_cast<int>(cudaMemcpyFromSymbol(host, g_wave_trace, bytes < sizeof(g_wave_trace) ? bytes : sizeof(g_wave_trace)));
+}
+#endif
+
+cudaError_t launch_wave(const LaunchConfig& c, const TensorDesc* descs, const uint32_t* unit_tensor, const WaveDesc* waves,
+                        uint32_t n_waves, const StepParams& P, uint32_t* amax, uint32_t* amax_next, float* s_old,
+                        uint32_t* grid_counter, uint32_t* status, int grid_cap, cudaStream_t stream, bool with_errors) {
+    if (n_waves == 0) return cudaSuccess;
+    ECO_S_FMT(c.format, ECO_S_OPT(c.optimizer, ECO_S_RND(c.rounding, {
+        if (with_errors)
+            return launch_wave_one<F, O, R, true>(descs, unit_tensor, waves, n_waves, P, c.scale_kind, amax, amax_next, s_old,
+                                                  grid_counter, status, grid_cap, c.sm_count, stream);
+        return launch_wave_one<F, O, R, false>(descs, unit_tensor, waves, n_waves, P, c.scale_kind, amax, amax_next, s_old,
+                                               grid_counter, status, grid_cap, c.sm_count, stream);
+    })))
+    return cudaErrorInvalidValue;
+}
+
 // Self-test of the bounded wait: one warp waits on an mbarrier that nothing ever arrives on.  The wait
 // must give up after limit_cycles, record its code and let the kernel end normally.
 __global__ void eco_wait_selftest_kernel(uint32_t* status, long long limit_cycles) {
@@ -588,6 +989,26 @@ __global__ void eco_wait_selftest_kernel(uint32_t* status, long long limit_cycle
     }
     __syncthreads();
     mbar_wait(smem_addr(&bar), 0, status, 7u, limit_cycles);
+}
+
+// Self-test of the bounded grid barrier: two CTAs of 8 warps meet at a barrier that expects three arrivals.  The
+// wait must give up after limit_cycles, record code 6 and let the kernel end normally.
+__global__ void __launch_bounds__(kConsumerWarps * 32) eco_grid_wait_selftest_kernel(uint32_t* counter, uint32_t* status, long long limit_cycles) {
+    __shared__ __align__(8) uint64_t bar;
+    __shared__ uint32_t abort_flag;
+    if (threadIdx.x == 0) {
+        mbar_init(smem_addr(&bar), kConsumerWarps);
+        abort_flag = 0u;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+    uint32_t phase = 0u;
+    wave_grid_barrier(counter, gridDim.x + 1u, status, &abort_flag, smem_addr(&bar), phase, threadIdx.x & 31, limit_cycles);
+}
+
+cudaError_t launch_grid_wait_selftest(uint32_t* counter, uint32_t* status, long long limit_cycles, cudaStream_t stream) {
+    eco_grid_wait_selftest_kernel<<<2, kConsumerWarps * 32, 0, stream>>>(counter, status, limit_cycles);
+    return cudaGetLastError();
 }
 
 cudaError_t launch_wait_selftest(uint32_t* status, long long limit_cycles, cudaStream_t stream) {

@@ -25,7 +25,7 @@ ECO_ROUND_NEAREST, ECO_ROUND_STOCHASTIC = 0, 1
 ECO_INJECT_NONE, ECO_INJECT_ECO, ECO_INJECT_EXACT = 0, 1, 2
 
 EXPORTED = ("eco_create", "eco_step", "eco_step_ex", "eco_step_begin", "eco_amax_buffer", "eco_step_end", "eco_step_host", "eco_host_create", "eco_host_step", "eco_host_copies", "eco_host_destroy",
-            "eco_step_static", "eco_check", "eco_attach_error_buffers", "eco_selftest_wait", "eco_destroy", "eco_last_error", "eco_quantize", "eco_dequantize",
+            "eco_step_static", "eco_check", "eco_attach_error_buffers", "eco_selftest_wait", "eco_selftest_grid_wait", "eco_destroy", "eco_last_error", "eco_quantize", "eco_dequantize",
             "eco_set_option", "eco_num_launches", "eco_version")
 
 
@@ -105,6 +105,8 @@ def load_library() -> ctypes.CDLL:
         L.eco_attach_error_buffers.argtypes = [vp, ctypes.POINTER(vp), ctypes.c_size_t]
         L.eco_selftest_wait.restype = ctypes.c_int
         L.eco_selftest_wait.argtypes = [vp, i64, vp]
+        L.eco_selftest_grid_wait.restype = ctypes.c_int
+        L.eco_selftest_grid_wait.argtypes = [vp, i64, vp]
         L.eco_destroy.restype = ctypes.c_int
         L.eco_destroy.argtypes = [vp]
         L.eco_last_error.restype = ctypes.c_char_p
@@ -331,6 +333,11 @@ def eco_attach_error_buffers(handle: int, buffers) -> None:
 def eco_selftest_wait(handle: int, limit_cycles: int = 2_000_000, stream: int = 0) -> int:
     """Run the bounded-wait self-test; returns the status (ECO_ERR_TIMEOUT when the mechanism works)."""
     return load_library().eco_selftest_wait(handle, limit_cycles, stream)
+
+
+def eco_selftest_grid_wait(handle: int, limit_cycles: int = 2_000_000, stream: int = 0) -> int:
+    """Run the self-test of the bounded grid barrier; returns the status (ECO_ERR_TIMEOUT when the mechanism works)."""
+    return load_library().eco_selftest_grid_wait(handle, limit_cycles, stream)
 
 
 def eco_destroy(handle: int) -> None:

@@ -200,6 +200,13 @@ def c3_small() -> Workload:
     return replace(w, name=w.name + "_small")
 
 
+def c3_no_embedding(layers: int = 26) -> Workload:
+    """The layers of the Gemma-3-1B-shaped set without the embedding: every tensor is at most 88 MB of inputs, i.e. about
+    as large as the L2 (the embedding is 3.3 GB)."""
+    w = c3(layers=layers, vocab=0)
+    return replace(w, name=w.name + f"_layers{layers}_only")
+
+
 def c3_rowwise() -> Workload:
     """The Gemma-3-1B-shaped set with one FP8 scale per row: the granularity of the paper's own FP8 runs (Sec. 4.1)."""
     w = c3()
@@ -288,7 +295,7 @@ def c4_dense_small() -> Workload:
     return replace(w, name="c4_smoe_2mat_fp8_block128_adam_sr_all_routed_small", tensors=[replace(t, zero_grad=False) for t in w.tensors])
 
 
-BY_NAME = {"c1": c1, "c2": c2, "c3": c3, "c4": c4, "c5": c5, "c3r": c3_rowwise, "c5t": c5_tensorwise_adam, "c4g": lambda: c4(expert_mats=3), "c4d": c4_dense,
+BY_NAME = {"c3f": c3_no_embedding, "c3fs": lambda: c3_no_embedding(3), "c1": c1, "c2": c2, "c3": c3, "c4": c4, "c5": c5, "c3r": c3_rowwise, "c5t": c5_tensorwise_adam, "c4g": lambda: c4(expert_mats=3), "c4d": c4_dense,
            "c3s": c3_small, "c3rs": c3_rowwise_small, "c4s": c4_small, "c5s": c5_small,
            "c4mx": c4_mx, "c4mxs": c4_mx_small, "c4ds": c4_dense_small}
 

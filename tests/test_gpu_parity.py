@@ -409,6 +409,9 @@ def test_bounded_wait_expires_and_reports_without_hurting_the_context():
         stream = torch.cuda.current_stream().cuda_stream
         assert eco.eco_selftest_wait(dev.handle, 2_000_000, stream) == eco.ECO_ERR_TIMEOUT
         eco.eco_check(dev.handle, stream)                       # cleared again: no error
+        # the wait between CTAs (grid barrier of the single-launch per-tensor step): an arrival that never comes
+        assert eco.eco_selftest_grid_wait(dev.handle, 2_000_000, stream) == eco.ECO_ERR_TIMEOUT
+        eco.eco_check(dev.handle, stream)
         grads = [wl.gradient_bf16(w, t, 1) for t in w.tensors]
         dev.tensors[0].grad.view(torch.int16).copy_(torch.from_numpy(grads[0].view(np.int16)))
         dev.step(1)
@@ -870,3 +873,43 @@ def test_c4_whole_set_streaming_equals_direct_load():
 
 def test_c5_whole_set_streaming_equals_direct_load():
     _whole_set_stream_against_direct(wl.c5())
+
+
+@pytest.mark.parametrize("fmt,sdt,opt", [(wl.FP8_E4M3, wl.SCALE_F32, wl.ADAM), (wl.INT4, wl.SCALE_BF16, wl.SGDM),
+                                         (wl.FP8_E5M2, wl.SCALE_BF16, wl.ADAM)])
+def test_single_launch_per_tensor_step_in_many_waves(fmt, sdt, opt):
+    """Per-tensor scales in one cooperative launch (both passes of every wave, a bounded grid barrier in between),
+    forced on and cut into waves of 1 MiB of inputs: a tensor with more units than the grid can keep in its stages
+    (re-loads in pass 2), tensors of a single unit (most CTAs have nothing to do in that wave and only meet at the
+    barrier), a tensor whose last unit is short, and a ragged one on the direct-load pair beside it.  Chained steps,
+    weight decay, against the oracle bit for bit; then the same through eco_step_begin / eco_step_end."""
+    shapes = [(768, 4096), (1, 128), (33, 1024), (2, 4224), (640, 1024), (5, 200), (3, 384), (257, 128)]
+    w = _mini(fmt, wl.PER_TENSOR, sdt, opt, wl.SR, shapes)
+    eco.eco_set_option("fused_tensor", 1)
+    eco.eco_set_option("wave_bytes", 1 << 20)
+    try:
+        dev = DeviceState(w)
+        dev.init_from_host()
+        dev.create()
+    finally:
+        eco.eco_set_option("fused_tensor", 2)
+        eco.eco_set_option("wave_bytes", 100 << 20)
+    assert eco.eco_num_launches(dev.handle) == 3          # one cooperative launch + the pair for the ragged tensor
+    ora = OracleState(w)
+    stream = torch.cuda.current_stream().cuda_stream
+    try:
+        for step in range(1, 6):
+            dev.set_grads_from_host(step)
+            if step < 5:
+                dev.step(step, weight_decay=0.05 if step % 2 else 0.0)
+            else:                                                     # the two-launch form of the same context
+                eco.eco_step_begin(dev.handle, w.lr, w.beta1, w.beta2, w.eps, step, w.step_seed, 0.05, 1.0, stream)
+                eco.eco_step_end(dev.handle, stream)
+            ora.step(step, weight_decay=0.05 if step % 2 else 0.0)
+            torch.cuda.synchronize()
+            eco.eco_check(dev.handle, stream)
+            compare(dev, ora, f"step {step}")
+        for i in range(len(w.tensors)):
+            assert (_np(dev.tensors[i].m).view(np.int32) == ora.m[i].view(np.int32)).all()
+    finally:
+        dev.destroy()
