@@ -352,6 +352,9 @@ eco_status eco_dequantize(const eco_config* cfg, const void* w, const void* scal
  *                     2 (default) when the whole context is a single wave.  eco_step_begin / eco_step_end always
  *                     use two launches (the exchange sits between them)
  *   "wave_bytes"      input bytes of a wave (default 100 MiB; at least 1 MiB)
+ *   "row_cluster"     per-row scales only: 1 (default) steps matrix rows of 4224..16384 columns (whole 128-column
+ *                     segments) with thread-block clusters of 2..4 CTAs that share a row; 0 sends them to the
+ *                     one-CTA-per-row kernel
  * No option changes any result bit.  Errors: ECO_ERR_INVALID_ARG for an unknown name.
  */
 eco_status eco_set_option(const char* name, int64_t value);

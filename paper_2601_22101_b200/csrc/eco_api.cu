@@ -24,7 +24,7 @@ namespace {
 thread_local std::string g_thread_error;
 
 enum LaunchKind { KIND_BLOCK_FAST = 0, KIND_BLOCK_GENERIC = 1, KIND_TENSOR = 2, KIND_ROW = 3, KIND_TENSOR_STREAM = 4,
-                  KIND_ROW_STREAM = 5, KIND_TENSOR_WAVE = 6 };
+                  KIND_ROW_STREAM = 5, KIND_TENSOR_WAVE = 6, KIND_ROW_CLUSTER = 7 };
 
 struct Launch {
     int kind;
@@ -33,6 +33,7 @@ struct Launch {
     uint32_t n_units;
     size_t wave_offset = 0;   // KIND_TENSOR_WAVE: into d_waves
     uint32_t n_waves = 0;
+    int cluster = 1;          // KIND_ROW_CLUSTER: CTAs per cluster
 };
 
 // Options settable through eco_set_option before eco_create.
@@ -43,6 +44,7 @@ struct Options {
     int64_t ctas_per_sm = 0;       // persistent grid = ctas_per_sm * SM count; 0: the kernel's own residency (2 or 3)
     int64_t fused_tensor = 2;      // per-tensor scale: both passes in one cooperative launch, wave by wave: 0 = never (launch
                                    // pair), 1 = always, 2 = when the whole context is a single wave (see eco_create)
+    int64_t row_cluster = 1;       // per-row scale: 1 = rows of 33..128 segments run on thread-block clusters; 0 = one CTA per row
     int64_t wave_bytes = 100ll << 20;   // per-tensor scale, one launch: input bytes of a wave of tensors (about the L2 size)
 };
 Options g_options;
@@ -249,6 +251,7 @@ eco_status eco_set_option(const char* name, int64_t value) {
     if (!std::strcmp(name, "reverse_pass2")) { g_options.reverse_pass2 = value; return ECO_OK; }
     if (!std::strcmp(name, "use_stream")) { g_options.use_stream = value; return ECO_OK; }
     if (!std::strcmp(name, "fused_tensor")) { g_options.fused_tensor = value; return ECO_OK; }
+    if (!std::strcmp(name, "row_cluster")) { g_options.row_cluster = value; return ECO_OK; }
     if (!std::strcmp(name, "wave_bytes")) {
         if (value < (1 << 20)) return fail(nullptr, ECO_ERR_INVALID_ARG, "wave_bytes must be at least 1 MiB");
         g_options.wave_bytes = value;
@@ -362,6 +365,10 @@ eco_status eco_create(eco_ctx** out, const eco_config* cfg, const eco_tensor* te
             if (kind == KIND_ROW) {
                 d.n_blocks = static_cast<uint64_t>(tensors[members[k]].rows);
                 nu = d.n_blocks;
+            } else if (kind == KIND_ROW_CLUSTER) {
+                // one unit per matrix row; the CTAs of a cluster share its segments
+                d.n_blocks = static_cast<uint64_t>(tensors[members[k]].rows) * d.blocks_per_row;
+                nu = static_cast<uint64_t>(tensors[members[k]].rows);
             } else if (kind == KIND_ROW_STREAM) {
                 // a unit is as many whole matrix rows as fit 32 rows of 128 elements
                 d.n_blocks = static_cast<uint64_t>(tensors[members[k]].rows) * d.blocks_per_row;
@@ -395,13 +402,24 @@ eco_status eco_create(eco_ctx** out, const eco_config* cfg, const eco_tensor* te
         ok = add_launch(KIND_BLOCK_FAST, fast) && add_launch(KIND_BLOCK_GENERIC, generic);
         ctx->num_launches = static_cast<int>(ctx->launches.size());
     } else if (cfg->granularity == ECO_SCALE_PER_ROW) {
-        // matrix rows of whole 128-element rows, at most 32 of them, go to the streaming kernel
-        std::vector<size_t> fast, generic;
+        // Matrix rows made of whole 128-element segments go to the streaming kernel: up to 32 segments as whole rows
+        // per unit, up to 32 * 4 segments with a thread-block cluster of 2..4 CTAs per matrix row (one launch per
+        // cluster size); anything else to the one-CTA-per-row kernel.
+        std::vector<size_t> fast, generic, clustered[5];
+        const int64_t seg_max = eco::stream_unit_rows();
         for (size_t i = 0; i < n; ++i) {
-            const bool streams = use_stream && tensors[i].cols % 128 == 0 && tensors[i].cols / 128 <= eco::stream_unit_rows();
-            (streams ? fast : generic).push_back(i);
+            const int64_t segs = tensors[i].cols / 128;
+            if (!use_stream || tensors[i].cols % 128 != 0 || segs > seg_max * eco::stream_max_cluster()) generic.push_back(i);
+            else if (segs <= seg_max) fast.push_back(i);
+            else if (g_options.row_cluster == 0) generic.push_back(i);
+            else clustered[(segs + seg_max - 1) / seg_max].push_back(i);
         }
-        ok = add_launch(KIND_ROW_STREAM, fast) && add_launch(KIND_ROW, generic);
+        ok = add_launch(KIND_ROW_STREAM, fast);
+        for (int c = 2; c <= eco::stream_max_cluster() && ok; ++c) {
+            ok = add_launch(KIND_ROW_CLUSTER, clustered[c]);
+            if (ok && !clustered[c].empty()) ctx->launches.back().cluster = c;
+        }
+        ok = ok && add_launch(KIND_ROW, generic);
         ctx->num_launches = static_cast<int>(ctx->launches.size());
     } else if (use_stream && cooperative && g_options.l2_group_bytes == 0 &&
                (g_options.fused_tensor == 1 || (g_options.fused_tensor == 2 && context_in_bytes <= static_cast<double>(g_options.wave_bytes)))) {
@@ -636,6 +654,11 @@ eco_status enqueue_step(eco_ctx* ctx, const StepParams& P, void* cuda_stream, in
             case KIND_ROW:
                 ECO_CUDA(ctx, eco::launch_row(ctx->lc, descs, units, L.n_units, P, stream));
                 break;
+            case KIND_ROW_CLUSTER:
+                ECO_CUDA(ctx, eco::launch_stream(ctx->lc, eco::STREAM_ROW, descs, units, L.n_units, P, nullptr, nullptr,
+                                                 nullptr, false, ctx->d_tickets, ctx->d_status, ctx->grid_cap, stream,
+                                                 ctx->has_error_buffers, L.cluster));
+                break;
             case KIND_ROW_STREAM:
                 ECO_CUDA(ctx, eco::launch_stream(ctx->lc, eco::STREAM_ROW, descs, units, L.n_units, P, nullptr, nullptr,
                                                  nullptr, false, ctx->d_tickets, ctx->d_status, ctx->grid_cap, stream, ctx->has_error_buffers));
@@ -665,7 +688,7 @@ eco_status eco_check(eco_ctx* ctx, void* cuda_stream) {
     if (code != 0)
         return fail(ctx, ECO_ERR_TIMEOUT, "a bounded wait inside a kernel expired (code %u: 1 = producer waiting for a free "
                     "stage, 2 = producer draining its copies, 3 = consumer waiting for data, 4/5 = per-row exchange, 6 = grid barrier of the "
-                    "single-launch per-tensor step, 7 = self-test, 8 = consumer warps meeting)", code);
+                    "single-launch per-tensor step, 7 = self-test, 8 = consumer warps meeting, 9 = row maximum from the cluster's peers)", code);
     return ECO_OK;
 }
 

@@ -36,7 +36,11 @@ enum : int { MODE_BLOCK = STREAM_BLOCK, MODE_TENSOR_AMAX = STREAM_TENSOR_AMAX, M
 cudaError_t launch_stream(const LaunchConfig& c, int mode, const TensorDesc* descs, const uint32_t* unit_tensor,
                           uint32_t n_units, const StepParams& P, uint32_t* amax, uint32_t* amax_next, float* s_old,
                           bool reverse, uint32_t* tickets, uint32_t* status, int grid_cap, cudaStream_t stream,
-                          bool with_errors = false);
+                          bool with_errors = false, int cluster = 1);
+// cluster > 1 (STREAM_ROW only): the units are single matrix rows of up to 32 * cluster segments of 128 columns; the
+// launch runs thread-block clusters of that many CTAs, each CTA streaming its slice of the row, the row maximum
+// exchanged through distributed shared memory (TensorDesc::n_blocks = rows * segments, one unit per matrix row).
+int stream_max_cluster();
 
 // A wave of the single-launch per-tensor step: the units [first_unit, first_unit + n_units) of the launch's unit table,
 // made of whole tensors.

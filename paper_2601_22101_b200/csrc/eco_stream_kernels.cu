@@ -71,7 +71,10 @@ struct StageLayout {
     static constexpr int kBarriers = 512;                        // 2 * kStages + 2 mbarriers, padded to 128; then the
                                                                  // per-row exchange: 32 maxima, 32 scales, 32 inverses
     static constexpr int kRowBars = 64;                          // two mbarriers of the per-row exchange
+    static constexpr int kPeerMax = 32;                          // per-row mode in a cluster: 2 x 4 partial row maxima from the peers
+    static constexpr int kClusterBars = 96;                      // ... and the two mbarriers the peers arrive on
     static constexpr int kExchange = 128;
+    static_assert(2 * kStages * 8 <= kPeerMax, "the stage barriers end before the cluster exchange area");
     static constexpr int kSmem = kBarriers + kStages * kBytes;
     static_assert(kBytes % 128 == 0, "stages stay 128-byte aligned");
 };
@@ -134,6 +137,37 @@ __device__ __forceinline__ void store_u16_first(void* p, uint32_t v, uint64_t po
     asm volatile("st.global.L2::cache_hint.u16 [%0], %1, %2;" ::"l"(p), "h"(static_cast<uint16_t>(v)), "l"(policy) : "memory");
 }
 
+// ---- thread-block cluster primitives (per-row scales on rows longer than one unit) ----
+__device__ __forceinline__ uint32_t cluster_rank() { uint32_t r; asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r)); return r; }
+__device__ __forceinline__ uint32_t cluster_size() { uint32_t r; asm volatile("mov.u32 %0, %%cluster_nctarank;" : "=r"(r)); return r; }
+// Address of the same shared-memory location in CTA `rank` of this cluster.
+__device__ __forceinline__ uint32_t peer_addr(uint32_t local, uint32_t rank) {
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(local), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ void peer_store_f32(uint32_t addr, float v) {
+    asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(addr), "f"(v) : "memory");
+}
+// Arrival on a peer's mbarrier; release at cluster scope orders this thread's earlier peer stores before it.
+__device__ __forceinline__ void peer_mbar_arrive(uint32_t addr) {
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(addr) : "memory");
+}
+// Bounded wait on an own mbarrier that peers arrive on (acquire at cluster scope).
+__device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity, uint32_t* status, uint32_t code) {
+    const long long t0 = clock64();
+    for (;;) {
+        uint32_t ok;
+        asm volatile("{ .reg .pred p; mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2; selp.u32 %0, 1, 0, p; }"
+                     : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+        if (ok) return true;
+        if (clock64() - t0 > kWaitLimitCycles) {
+            atomicExch(status, code);
+            return false;
+        }
+    }
+}
+
 // max |x| over the 32 lanes in one instruction (sm_100a warp reduction on binary32; NaN operands are
 // ignored, as by fmaxf).  Every lane receives the result.  The final maximum with zero makes a warp whose
 // operands are ALL NaN return 0 (a block of nothing but NaN has no maximum: it takes the scale of an all-zero block).
@@ -151,6 +185,12 @@ __device__ __forceinline__ uint32_t units_of(const TensorDesc& T) {
 // elements 4l..4l+3 of each.  FULL: all 32 rows are present (every unit but the last of a tensor).
 // TS: the scales of the per-tensor modes (old scale for the dequantization; new scale and its inverse for pass 2).
 struct TensorScales { float s_old, s_new, inv_new; };
+// Per-row mode inside a thread-block cluster: this CTA's rank, the cluster's size (1 = no cluster), the shared-memory
+// addresses of the exchange slots and barriers, and the phase parity of the barrier this unit uses.
+struct ClusterInfo {
+    uint32_t rank, size, peer_max, bars, phase;
+    const float* peer_max_ptr;
+};
 // HINT: stores carry an evict-first hint (`store_policy`); false = plain stores.
 template <int FMT, int OPT, int RND, int MODE, bool FULL, bool ERR, int NS = 4, bool HINT = false>
 __device__ __forceinline__ bool consume_unit(const StepParams& P, const int scale_kind, const uint8_t* st,
@@ -159,7 +199,8 @@ __device__ __forceinline__ bool consume_unit(const StepParams& P, const int scal
                                              float& run_max, float* xchg, const uint32_t row_bars,
                                              const uint32_t row_parity, uint32_t* status,
                                              const TensorScales ts = TensorScales{1.0f, 1.0f, 1.0f},
-                                             const uint64_t store_policy = 0) {
+                                             const uint64_t store_policy = 0,
+                                             const ClusterInfo cl = ClusterInfo{0u, 1u, 0u, 0u, 0u, nullptr}) {
     using SL = StageLayout<FMT, OPT>;
     // Row (of 128 elements) behind slot k of this warp.  Per-row mode deals the rows round-robin (warp, warp + 8, ...)
     // so that a unit of fewer than 32 rows leaves every warp with 3 or 4 rows instead of some with none; NS is the
@@ -307,14 +348,32 @@ __device__ __forceinline__ bool consume_unit(const StepParams& P, const int scal
         if (!mbar_wait(row_bars, row_parity, status, 4u)) return false;
         for (uint32_t j = static_cast<uint32_t>(warp); j < n_mrows; j += kConsumerWarps) {
             const float x = static_cast<uint32_t>(lane) < seg_per_row ? xmax[j * seg_per_row + lane] : 0.0f;
-            const float a = warp_amax(x);
+            float a = warp_amax(x);
+            bool owner = true;
+            if (cl.size > 1) {
+                // A matrix row longer than one unit: the CTAs of the cluster each hold a slice of it (this unit is ONE
+                // matrix row, so j == 0 and only warp 0 is here).  Lane r hands this CTA's partial maximum to CTA r --
+                // a store into its shared memory, then an arrival on its mbarrier -- and the warp waits, bounded, for
+                // the arrivals of all CTAs on its own.  Slots and barriers alternate with the unit's parity, so a
+                // CTA that is a unit ahead cannot disturb one that is still reading.
+                const uint32_t slot = cl.peer_max + (row_parity * 4u + cl.rank) * 4u;
+                const uint32_t bar = cl.bars + row_parity * 8u;
+                if (static_cast<uint32_t>(lane) < cl.size) {
+                    peer_store_f32(peer_addr(slot, lane), a);
+                    peer_mbar_arrive(peer_addr(bar, lane));
+                }
+                if (!mbar_wait_cluster(bar, cl.phase, status, 9u)) return false;
+                const float* pm = cl.peer_max_ptr + row_parity * 4u;
+                a = warp_amax(static_cast<uint32_t>(lane) < cl.size ? pm[lane] : 0.0f);
+                owner = cl.rank == 0u;
+            }
             float s_j, inv_j;
             uint32_t bits_j;
             make_scale_div<FMT>(a, scale_kind == SCALE_KIND_BF16, s_j, inv_j, bits_j);
             if (lane == 0) {
                 xs[j] = s_j;
                 xinv[j] = inv_j;
-                store_scale(sp, mrow0 + j, scale_kind, s_j, bits_j);
+                if (owner) store_scale(sp, mrow0 + j, scale_kind, s_j, bits_j);
             }
         }
         __syncwarp();
@@ -405,9 +464,17 @@ eco_stream_kernel(const TensorDesc* __restrict__ descs, const uint32_t* __restri
         }
         mbar_init(row_bars, kConsumerWarps);
         mbar_init(row_bars + 8, kConsumerWarps);
+        mbar_init(smem_addr(smem + SL::kClusterBars), cluster_size());
+        mbar_init(smem_addr(smem + SL::kClusterBars + 8), cluster_size());
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
+    const uint32_t csize = MODE == MODE_ROW ? cluster_size() : 1u, crank = MODE == MODE_ROW ? cluster_rank() : 0u;
+    if (csize > 1) {
+        // peers arrive on this CTA's barriers: nobody starts before every CTA of the cluster has initialised its own
+        asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+        asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+    }
 
     if (warp == kConsumerWarps) {
         // ------------------------------ producer ------------------------------
@@ -424,28 +491,36 @@ eco_stream_kernel(const TensorDesc* __restrict__ descs, const uint32_t* __restri
             if (lane == 0) t = atomicAdd(tickets, 1u);
             return __shfl_sync(0xFFFFFFFFu, t, 0);
         };
-        uint32_t ticket = draw();
         uint32_t it = 0;
         bool ok = true;
-        while (ticket < n_tickets) {
-            const uint32_t next_ticket = draw();          // in flight while this unit is set up
-            const uint32_t cand = (ticket % W) * per_region + ticket / W;
-            ticket = next_ticket;
-            if (cand >= n_units) continue;
-            const uint32_t unit = reverse ? (n_units - 1 - cand) : cand;
+        // Stages one unit: waits for a free stage, issues the copies, writes the header.
+        auto stage_unit = [&](const uint32_t unit) -> bool {
             const TensorDesc T = descs[__ldg(unit_tensor + unit)];
             const uint32_t s = it % S, ph = (it / S) & 1;
-            ok = mbar_wait(empty0 + 8 * s, ph ^ 1, status, 1u);
-            if (!ok) break;
+            if (!mbar_wait(empty0 + 8 * s, ph ^ 1, status, 1u)) return false;
             uint8_t* st = stage0 + static_cast<size_t>(s) * SL::kBytes;
             const uint32_t local = unit - T.first_unit;
-            const uint32_t unit_rows = MODE == MODE_ROW ? T.unit_rows : static_cast<uint32_t>(kUnitRows);
-            const uint64_t row0 = static_cast<uint64_t>(local) * unit_rows;
-            const uint64_t left = T.n_blocks - row0;
-            const uint32_t nrows = left < unit_rows ? static_cast<uint32_t>(left) : unit_rows;
-            const uint32_t mrows_per_unit = MODE == MODE_ROW ? unit_rows / T.blocks_per_row : 0u;
-            const uint64_t mrow0 = static_cast<uint64_t>(local) * mrows_per_unit;
-            const uint32_t n_mrows = MODE == MODE_ROW ? nrows / T.blocks_per_row : 0u;
+            uint64_t row0, mrow0;
+            uint32_t nrows, n_mrows, segs;
+            if (MODE == MODE_ROW && csize > 1) {
+                // the unit is ONE matrix row of R segments; this CTA takes segments [rank Rc, (rank + 1) Rc) of it
+                const uint32_t R = T.blocks_per_row, Rc = div_ceil_u32(R, csize);
+                const uint32_t lo = crank * Rc, hi = lo + Rc < R ? lo + Rc : R;
+                row0 = static_cast<uint64_t>(local) * R + lo;
+                nrows = hi - lo;
+                mrow0 = local;
+                n_mrows = 1u;
+                segs = nrows;
+            } else {
+                const uint32_t unit_rows = MODE == MODE_ROW ? T.unit_rows : static_cast<uint32_t>(kUnitRows);
+                row0 = static_cast<uint64_t>(local) * unit_rows;
+                const uint64_t left = T.n_blocks - row0;
+                nrows = left < unit_rows ? static_cast<uint32_t>(left) : unit_rows;
+                const uint32_t mrows_per_unit = MODE == MODE_ROW ? unit_rows / T.blocks_per_row : 0u;
+                mrow0 = static_cast<uint64_t>(local) * mrows_per_unit;
+                n_mrows = MODE == MODE_ROW ? nrows / T.blocks_per_row : 0u;
+                segs = T.blocks_per_row;
+            }
             const uint32_t full = full0 + 8 * s;
             if (lane == 0) {
                 const uint32_t cb = nrows * SL::kCodeRow, gb = nrows * 256u, mb = nrows * 512u;
@@ -458,7 +533,7 @@ eco_stream_kernel(const TensorDesc* __restrict__ descs, const uint32_t* __restri
                 h.w = T.w; h.scale = T.scale; h.m = T.m; h.v = T.v;
                 h.row0 = row0; h.nrows = nrows; h.tensor_id = T.tensor_id; h.slot = T.slot;
                 h.s_old = 1.0f; h.s_new = 1.0f; h.inv_new = 1.0f;
-                h.seg_per_row = T.blocks_per_row; h.div_magic = 65536u / T.blocks_per_row + 1u;
+                h.seg_per_row = segs; h.div_magic = 65536u / segs + 1u;
                 h.n_mrows = n_mrows; h.pass = 0u; h.barrier_target = 0u; h.first_of_tensor = 0u; h.mrow0 = mrow0; h.index_base = T.index_base; h.e = T.e;
                 if (MODE == MODE_TENSOR_AMAX) {
                     h.s_old = load_scale(T.scale, 0, scale_kind);
@@ -488,10 +563,27 @@ eco_stream_kernel(const TensorDesc* __restrict__ descs, const uint32_t* __restri
             __syncwarp();
             if (lane == 0) mbar_arrive(full);
             ++it;
-        }
-        if (lane == 0 && atomicAdd(tickets + 1, 1u) == gridDim.x - 1) {
-            tickets[0] = 0u;                               // every CTA has drawn its last ticket
-            tickets[1] = 0u;
+            return true;
+        };
+        if (MODE == MODE_ROW && csize > 1) {
+            // a cluster works on one matrix row at a time, all its CTAs on the same one: cluster c of K takes the
+            // rows c, c + K, ... of the launch (no tickets: the CTAs of a cluster must agree without talking)
+            const uint32_t n_clusters = gridDim.x / csize, cid = blockIdx.x / csize;
+            for (uint32_t unit = cid; unit < n_units && ok; unit += n_clusters) ok = stage_unit(unit);
+        } else {
+            uint32_t ticket = draw();
+            while (ticket < n_tickets) {
+                const uint32_t next_ticket = draw();          // in flight while this unit is set up
+                const uint32_t cand = (ticket % W) * per_region + ticket / W;
+                ticket = next_ticket;
+                if (cand >= n_units) continue;
+                ok = stage_unit(reverse ? (n_units - 1 - cand) : cand);
+                if (!ok) break;
+            }
+            if (lane == 0 && atomicAdd(tickets + 1, 1u) == gridDim.x - 1) {
+                tickets[0] = 0u;                               // every CTA has drawn its last ticket
+                tickets[1] = 0u;
+            }
         }
         if (ok) {
             // end marker: a stage whose header says "no rows"
@@ -530,15 +622,19 @@ eco_stream_kernel(const TensorDesc* __restrict__ descs, const uint32_t* __restri
         if constexpr (MODE == MODE_ROW) {
             // rows are dealt round-robin: this warp has rows warp, warp + 8, ... below nrows
             const int mine = static_cast<int>(nrows) > warp ? (static_cast<int>(nrows) - warp + kConsumerWarps - 1) / kConsumerWarps : 0;
+            // (in a cluster: unit `it` uses exchange slot and barrier it & 1, whose phase parity is (it >> 1) & 1)
+            const ClusterInfo cl{crank, csize, smem_addr(smem + SL::kPeerMax), smem_addr(smem + SL::kClusterBars), (it >> 1) & 1u,
+                                 reinterpret_cast<const float*>(smem + SL::kPeerMax)};
+            const TensorScales none{1.0f, 1.0f, 1.0f};
             if (mine == 4)
                 ok = consume_unit<FMT, OPT, RND, MODE, true, ERR, 4>(P, scale_kind, st, h, empty, warp, lane, scratch_amax, cur_slot,
-                                                                     run_max, xchg, row_bars, it & 1u, status);
+                                                                     run_max, xchg, row_bars, it & 1u, status, none, 0, cl);
             else if (mine == 3)
                 ok = consume_unit<FMT, OPT, RND, MODE, true, ERR, 3>(P, scale_kind, st, h, empty, warp, lane, scratch_amax, cur_slot,
-                                                                     run_max, xchg, row_bars, it & 1u, status);
+                                                                     run_max, xchg, row_bars, it & 1u, status, none, 0, cl);
             else
                 ok = consume_unit<FMT, OPT, RND, MODE, false, ERR, 4>(P, scale_kind, st, h, empty, warp, lane, scratch_amax, cur_slot,
-                                                                      run_max, xchg, row_bars, it & 1u, status);
+                                                                      run_max, xchg, row_bars, it & 1u, status, none, 0, cl);
         } else if (nrows == kUnitRows)   // (discarded statement of the if constexpr above for the per-row mode)
             ok = consume_unit<FMT, OPT, RND, MODE, true, ERR>(P, scale_kind, st, h, empty, warp, lane, scratch_amax, cur_slot,
                                                               run_max, xchg, row_bars, it & 1u, status,
@@ -901,7 +997,8 @@ static cudaError_t launch_wave_one(const TensorDesc* descs, const uint32_t* unit
 template <int FMT, int OPT, int RND, int MODE, bool ERR = false>
 static cudaError_t launch_one(const TensorDesc* descs, const uint32_t* unit_tensor, uint32_t n_units, const StepParams& P,
                               int scale_kind, uint32_t* amax, uint32_t* amax_next, float* s_old, bool reverse,
-                              uint32_t* tickets, uint32_t* status, int grid_cap, int sm_count, cudaStream_t stream) {
+                              uint32_t* tickets, uint32_t* status, int grid_cap, int sm_count, cudaStream_t stream,
+                              int cluster = 1) {
     using SL = StageLayout<FMT, OPT>;
     static bool configured = false;
     auto kernel = eco_stream_kernel<FMT, OPT, RND, MODE, ERR>;
@@ -911,10 +1008,31 @@ static cudaError_t launch_one(const TensorDesc* descs, const uint32_t* unit_tens
         configured = true;
     }
     const uint32_t cap = static_cast<uint32_t>(grid_cap > 0 ? grid_cap : sm_count * stream_ctas_per_sm<OPT, ERR>());
+    const int interleave = (MODE == MODE_BLOCK || MODE == MODE_BLOCK32 || MODE == MODE_ROW) ? kInterleave : 1;
+    if (cluster > 1) {
+        // per-row scales on rows of several units: clusters of `cluster` CTAs, one matrix row per cluster at a time
+        const uint32_t c = static_cast<uint32_t>(cluster);
+        uint32_t n_clusters = cap / c;
+        if (n_clusters > n_units) n_clusters = n_units;
+        if (n_clusters == 0) return cudaErrorInvalidConfiguration;
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(n_clusters * c);
+        cfg.blockDim = dim3(kStreamThreads);
+        cfg.dynamicSmemBytes = SL::kSmem;
+        cfg.stream = stream;
+        cudaLaunchAttribute attr;
+        attr.id = cudaLaunchAttributeClusterDimension;
+        attr.val.clusterDim.x = c;
+        attr.val.clusterDim.y = 1;
+        attr.val.clusterDim.z = 1;
+        cfg.attrs = &attr;
+        cfg.numAttrs = 1;
+        return cudaLaunchKernelEx(&cfg, kernel, descs, unit_tensor, n_units, P, scale_kind, amax, amax_next, s_old,
+                                  reverse ? 1 : 0, interleave, tickets, status);
+    }
     const uint32_t grid = n_units < cap ? n_units : cap;
     kernel<<<grid, kStreamThreads, SL::kSmem, stream>>>(descs, unit_tensor, n_units, P, scale_kind, amax, amax_next,
-                                                        s_old, reverse ? 1 : 0,
-                                                        (MODE == MODE_BLOCK || MODE == MODE_BLOCK32 || MODE == MODE_ROW) ? kInterleave : 1, tickets, status);
+                                                        s_old, reverse ? 1 : 0, interleave, tickets, status);
     return cudaGetLastError();
 }
 
@@ -932,7 +1050,7 @@ static cudaError_t launch_one(const TensorDesc* descs, const uint32_t* unit_tens
 cudaError_t launch_stream(const LaunchConfig& c, int mode, const TensorDesc* descs, const uint32_t* unit_tensor,
                           uint32_t n_units, const StepParams& P, uint32_t* amax, uint32_t* amax_next, float* s_old,
                           bool reverse, uint32_t* tickets, uint32_t* status, int grid_cap, cudaStream_t stream,
-                          bool with_errors) {
+                          bool with_errors, int cluster) {
     if (n_units == 0) return cudaSuccess;
     if (mode == STREAM_TENSOR_AMAX) {
         ECO_S_FMT(c.format, ECO_S_OPT(c.optimizer, {
@@ -942,7 +1060,7 @@ cudaError_t launch_stream(const LaunchConfig& c, int mode, const TensorDesc* des
     }
 #define ECO_S_LAUNCH(MODE_, ERR_)                                                                                      \
     return launch_one<F, O, R, MODE_, ERR_>(descs, unit_tensor, n_units, P, c.scale_kind, amax, amax_next, s_old, reverse, \
-                                            tickets, status, grid_cap, c.sm_count, stream)
+                                            tickets, status, grid_cap, c.sm_count, stream, MODE_ == MODE_ROW ? cluster : 1)
     ECO_S_FMT(c.format, ECO_S_OPT(c.optimizer, ECO_S_RND(c.rounding, {
         if (with_errors) {
             if (mode == STREAM_ROW) ECO_S_LAUNCH(MODE_ROW, true);
@@ -1017,5 +1135,6 @@ cudaError_t launch_wait_selftest(uint32_t* status, long long limit_cycles, cudaS
 }
 
 int stream_unit_rows() { return kUnitRows; }
+int stream_max_cluster() { return 4; }
 
 }  // namespace eco

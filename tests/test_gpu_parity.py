@@ -517,8 +517,12 @@ def test_row_shards_with_amax_exchange_equal_the_unsplit_step(fmt, opt, sdt):
                                          (wl.FP8_E4M3, wl.SCALE_BF16, wl.SGDM)])
 def test_per_row_scales_on_long_and_short_rows(fmt, sdt, opt):
     """Per-row scales over the kernels that serve them: rows of up to 4096 columns made of whole 128-element
-    segments (streaming kernel, several matrix rows per unit), longer or ragged rows (one CTA per row)."""
-    shapes = [(5, 6912), (3, 12288), (2, 4224), (70, 1152), (9, 4096), (40, 128), (3, 8190), (4, 200)]
+    segments (streaming kernel, several matrix rows per unit); rows of up to 16384 columns (clusters of 2, 3 or 4
+    CTAs share a matrix row and exchange its maximum through distributed shared memory: 4224 and 6912 and 8192
+    columns with pairs, 12288 and 12416 with three, 16384 with four CTAs; more rows than clusters, so that every
+    cluster takes several); longer or ragged rows (one CTA per row)."""
+    shapes = [(5, 6912), (3, 12288), (2, 4224), (70, 1152), (9, 4096), (40, 128), (3, 8190), (4, 200),
+              (601, 8192), (2, 16384), (1, 16512), (300, 12416)]
     run_chained(_mini(fmt, wl.PER_ROW, sdt, opt, wl.SR, shapes), steps=5)
 
 
