@@ -64,6 +64,7 @@ struct eco_ctx {
     uint32_t* d_tickets = nullptr;
     eco::WaveDesc* d_waves = nullptr;
     uint32_t* d_grid_counter = nullptr;
+    uint32_t* d_wave_tickets = nullptr;   // two per wave; NULL for a single wave (static split)
     bool pending = false;          // eco_step_begin issued, eco_step_end not yet
     std::vector<TensorDesc> h_descs;      // host copy of the descriptor table (patched by eco_attach_error_buffers)
     std::vector<size_t> desc_of_tensor;   // tensor index -> its descriptor
@@ -534,6 +535,10 @@ eco_status eco_create(eco_ctx** out, const eco_config* cfg, const eco_tensor* te
         ECO_CUDA_CTX(cudaMemcpy(ctx->d_waves, waves.data(), waves.size() * sizeof(eco::WaveDesc), cudaMemcpyHostToDevice));
         ECO_CUDA_CTX(cudaMalloc(&ctx->d_grid_counter, 2 * sizeof(uint32_t)));
         ECO_CUDA_CTX(cudaMemset(ctx->d_grid_counter, 0, 2 * sizeof(uint32_t)));
+        if (waves.size() > 1) {
+            ECO_CUDA_CTX(cudaMalloc(&ctx->d_wave_tickets, 2 * waves.size() * sizeof(uint32_t)));
+            ECO_CUDA_CTX(cudaMemset(ctx->d_wave_tickets, 0, 2 * waves.size() * sizeof(uint32_t)));
+        }
     }
     ECO_CUDA_CTX(cudaDeviceSynchronize());
 #undef ECO_CUDA_CTX
@@ -638,7 +643,9 @@ eco_status enqueue_step(eco_ctx* ctx, const StepParams& P, void* cuda_stream, in
                 if (pass == PASS_BOTH) {
                     ECO_CUDA(ctx, eco::launch_wave(ctx->lc, descs, units, ctx->d_waves + L.wave_offset, L.n_waves, P,
                                                    ctx->d_amax[parity], ctx->d_amax[parity ^ 1], ctx->d_s_old,
-                                                   ctx->d_grid_counter, ctx->d_status, ctx->grid_cap, stream, ctx->has_error_buffers));
+                                                   ctx->d_grid_counter,
+                                                   ctx->d_wave_tickets ? ctx->d_wave_tickets + 2 * L.wave_offset : nullptr,
+                                                   ctx->d_status, ctx->grid_cap, stream, ctx->has_error_buffers));
                     break;
                 }
                 // the step cut in two for an amax exchange between ranks: the two passes as separate launches
@@ -747,6 +754,7 @@ eco_status eco_destroy(eco_ctx* ctx) {
     cudaFree(ctx->d_tickets);
     cudaFree(ctx->d_waves);
     cudaFree(ctx->d_grid_counter);
+    cudaFree(ctx->d_wave_tickets);
     delete ctx;
     return ECO_OK;
 }

@@ -49,11 +49,15 @@ struct WaveDesc {
 };
 
 // Per-tensor scales in one cooperative launch (see eco_wave_kernel): both passes of every wave, a grid barrier in
-// between.  `grid_counter`: two device words, zero before the first launch, rewound by the kernel itself.  The grid is
-// the number of CTAs the device can hold at once (or grid_cap, if that is smaller).
+// between.  `grid_counter`: two device words, zero before the first launch, rewound by the kernel itself.
+// `wave_tickets`: NULL = every CTA owns a fixed share of each wave (what it streamed in pass 1 is still in its
+// shared memory for pass 2: the form for a single wave); else 2 * n_waves device words, zero before the first launch
+// and rewound by the kernel, from which the units of each pass are handed out.  The grid is the number of CTAs the
+// device can hold at once (or grid_cap, if that is smaller).
 cudaError_t launch_wave(const LaunchConfig& c, const TensorDesc* descs, const uint32_t* unit_tensor, const WaveDesc* waves,
                         uint32_t n_waves, const StepParams& P, uint32_t* amax, uint32_t* amax_next, float* s_old,
-                        uint32_t* grid_counter, uint32_t* status, int grid_cap, cudaStream_t stream, bool with_errors);
+                        uint32_t* grid_counter, uint32_t* wave_tickets, uint32_t* status, int grid_cap, cudaStream_t stream,
+                        bool with_errors);
 
 // One warp waits, for at most limit_cycles, on a barrier nothing arrives on; then writes code 7 to *status.
 cudaError_t launch_wait_selftest(uint32_t* status, long long limit_cycles, cudaStream_t stream);

@@ -733,7 +733,8 @@ __global__ void __launch_bounds__(kStreamThreads, stream_ctas_per_sm<OPT, ERR>()
 eco_wave_kernel(const TensorDesc* __restrict__ descs, const uint32_t* __restrict__ unit_tensor,
                 const WaveDesc* __restrict__ waves, const uint32_t n_waves, const StepParams P, const int scale_kind,
                 uint32_t* __restrict__ scratch_amax, uint32_t* __restrict__ scratch_amax_next,
-                float* __restrict__ scratch_s_old, uint32_t* __restrict__ grid_counter, uint32_t* __restrict__ status) {
+                float* __restrict__ scratch_s_old, uint32_t* __restrict__ grid_counter, uint32_t* __restrict__ wave_tickets,
+                uint32_t* __restrict__ status) {
     using SL = StageLayout<FMT, OPT>;
     constexpr int S = SL::kStages;
     extern __shared__ __align__(128) uint8_t smem[];
@@ -741,6 +742,7 @@ eco_wave_kernel(const TensorDesc* __restrict__ descs, const uint32_t* __restrict
     const uint32_t full0 = smem_addr(bars), empty0 = smem_addr(bars + S);
     uint8_t* stage0 = smem + SL::kBarriers;
     uint32_t* abort_flag = reinterpret_cast<uint32_t*>(smem + SL::kExchange);
+    const bool dynamic = wave_tickets != nullptr;
     const uint32_t sync_bar = smem_addr(smem + SL::kRowBars);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -836,7 +838,37 @@ eco_wave_kernel(const TensorDesc* __restrict__ descs, const uint32_t* __restrict
             ++it;
             return true;
         };
-        for (uint32_t w = 0; w < n_waves && ok; ++w) {
+        // Several waves: the units of each pass of a wave are handed out by a ticket counter (two per wave), so that
+        // every CTA is busy until the pass runs dry and all reach the barrier together; pass 2 walks the wave newest
+        // first and finds it in L2.  (With the static split below, CTAs that are a little slower -- or hold one unit
+        // more -- keep the whole grid waiting at every barrier.)
+        auto draw = [&](uint32_t* counter) -> uint32_t {
+            uint32_t t = 0;
+            if (lane == 0) t = atomicAdd(counter, 1u);
+            return __shfl_sync(0xFFFFFFFFu, t, 0);
+        };
+        for (uint32_t w = 0; dynamic && w < n_waves && ok; ++w) {
+            const uint32_t first = waves[w].first_unit, n = waves[w].n_units;
+            uint32_t t = draw(wave_tickets + 2 * w);
+            while (t < n && ok) {
+                const uint32_t tn = draw(wave_tickets + 2 * w);           // in flight while this unit is staged
+                ok = publish(WAVE_AMAX, first + t, true, false, 0u);
+                t = tn;
+            }
+            if (!ok) break;
+            const uint32_t target = (w + 1u) * G;
+            t = draw(wave_tickets + 2 * w + 1);
+            if (t >= n) ok = publish(WAVE_NOOP, 0u, false, false, target);   // nothing left for this CTA: only the barrier
+            bool first_pub = true;
+            while (t < n && ok) {
+                const uint32_t tn = draw(wave_tickets + 2 * w + 1);
+                ok = publish(WAVE_APPLY, first + (n - 1u - t), true, true, first_pub ? target : 0u);
+                first_pub = false;
+                t = tn;
+            }
+        }
+        // A single wave: static split, so that what a CTA streamed in pass 1 is still in its stages for pass 2.
+        for (uint32_t w = 0; !dynamic && w < n_waves && ok; ++w) {
             const uint32_t first = waves[w].first_unit, n = waves[w].n_units;
             const uint32_t mine = n > cta ? (n - cta + G - 1) / G : 0u;          // units first + cta + j G, j < mine
 #pragma unroll
@@ -965,13 +997,16 @@ eco_wave_kernel(const TensorDesc* __restrict__ descs, const uint32_t* __restrict
     if (threadIdx.x == 0 && atomicAdd(grid_counter + 1, 1u) == G - 1) {
         grid_counter[0] = 0u;
         grid_counter[1] = 0u;
+        if (dynamic)
+            for (uint32_t k = 0; k < 2u * n_waves; ++k) wave_tickets[k] = 0u;
     }
 }
 
 template <int FMT, int OPT, int RND, bool ERR>
 static cudaError_t launch_wave_one(const TensorDesc* descs, const uint32_t* unit_tensor, const WaveDesc* waves, uint32_t n_waves,
                                    const StepParams& P, int scale_kind, uint32_t* amax, uint32_t* amax_next, float* s_old,
-                                   uint32_t* grid_counter, uint32_t* status, int grid_cap, int sm_count, cudaStream_t stream) {
+                                   uint32_t* grid_counter, uint32_t* wave_tickets, uint32_t* status, int grid_cap, int sm_count,
+                                   cudaStream_t stream) {
     using SL = StageLayout<FMT, OPT>;
     static int resident = -1;                     // CTAs of this instantiation that fit one SM
     auto kernel = eco_wave_kernel<FMT, OPT, RND, ERR>;
@@ -989,7 +1024,7 @@ static cudaError_t launch_wave_one(const TensorDesc* descs, const uint32_t* unit
     if (grid_cap > 0 && grid_cap < grid) grid = grid_cap;
     StepParams Pc = P;
     int sk = scale_kind;
-    void* args[] = {&descs, &unit_tensor, &waves, &n_waves, &Pc, &sk, &amax, &amax_next, &s_old, &grid_counter, &status};
+    void* args[] = {&descs, &unit_tensor, &waves, &n_waves, &Pc, &sk, &amax, &amax_next, &s_old, &grid_counter, &wave_tickets, &status};
     return cudaLaunchCooperativeKernel(reinterpret_cast<void*>(kernel), dim3(grid), dim3(kStreamThreads), args, SL::kSmem, stream);
 }
 
@@ -1085,14 +1120,15 @@ extern "C" int eco_debug_read_wave_trace(void* host, size_t bytes) {
 
 cudaError_t launch_wave(const LaunchConfig& c, const TensorDesc* descs, const uint32_t* unit_tensor, const WaveDesc* waves,
                         uint32_t n_waves, const StepParams& P, uint32_t* amax, uint32_t* amax_next, float* s_old,
-                        uint32_t* grid_counter, uint32_t* status, int grid_cap, cudaStream_t stream, bool with_errors) {
+                        uint32_t* grid_counter, uint32_t* wave_tickets, uint32_t* status, int grid_cap, cudaStream_t stream,
+                        bool with_errors) {
     if (n_waves == 0) return cudaSuccess;
     ECO_S_FMT(c.format, ECO_S_OPT(c.optimizer, ECO_S_RND(c.rounding, {
         if (with_errors)
             return launch_wave_one<F, O, R, true>(descs, unit_tensor, waves, n_waves, P, c.scale_kind, amax, amax_next, s_old,
-                                                  grid_counter, status, grid_cap, c.sm_count, stream);
+                                                  grid_counter, wave_tickets, status, grid_cap, c.sm_count, stream);
         return launch_wave_one<F, O, R, false>(descs, unit_tensor, waves, n_waves, P, c.scale_kind, amax, amax_next, s_old,
-                                               grid_counter, status, grid_cap, c.sm_count, stream);
+                                               grid_counter, wave_tickets, status, grid_cap, c.sm_count, stream);
     })))
     return cudaErrorInvalidValue;
 }

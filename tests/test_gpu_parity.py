@@ -820,7 +820,7 @@ def _digest(buf: torch.Tensor):
     return out
 
 
-def _whole_set_stream_against_direct(w: wl.Workload, steps=2):
+def _whole_set_stream_against_direct(w: wl.Workload, steps=2, fused=None):
     """Every tensor of a full-size set, not a sample: the set is stepped by the persistent streaming kernels (ticket
     scheduler, the configuration the benchmark times) and again, from the same seeded state, by the direct-load
     kernels (one CTA per unit, no scheduler).  All codes, scales and moments must agree bit for bit: a unit that the
@@ -837,6 +837,8 @@ def _whole_set_stream_against_direct(w: wl.Workload, steps=2):
     results = []
     for use_stream in (1, 0):
         eco.eco_set_option("use_stream", use_stream)
+        if fused is not None:
+            eco.eco_set_option("fused_tensor", fused)
         try:
             dev = DeviceState(w)
             dev.init_on_device(seed=91)
@@ -844,6 +846,7 @@ def _whole_set_stream_against_direct(w: wl.Workload, steps=2):
             dev.create()
         finally:
             eco.eco_set_option("use_stream", 1)
+            eco.eco_set_option("fused_tensor", 2)
         try:
             for step in range(1, steps + 1):
                 dev.step(step)
@@ -869,6 +872,12 @@ def _whole_set_stream_against_direct(w: wl.Workload, steps=2):
 
 def test_c3_whole_set_streaming_equals_direct_load():
     _whole_set_stream_against_direct(wl.c3())
+
+
+def test_c3_whole_set_in_one_cooperative_launch_equals_direct_load():
+    """The same with the single-launch form of the per-tensor step forced on: 88 waves, both passes of each handed
+    out by tickets, a grid barrier per wave."""
+    _whole_set_stream_against_direct(wl.c3(), fused=1)
 
 
 def test_c4_whole_set_streaming_equals_direct_load():
