@@ -328,9 +328,7 @@ def main():
     args = ap.parse_args()
 
     if args.impl == "reference":
-        if args.steps == 20 and args.warmup == 5:
-            args.steps, args.warmup = 5, 1
-        run_reference(args)
+        run_reference(args)       # every step is a bounded sample (about 4 M parameters, 0.15 s on one core)
         return
 
     import torch

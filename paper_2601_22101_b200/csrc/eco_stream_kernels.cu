@@ -271,8 +271,13 @@ __device__ __forceinline__ bool consume_unit(const StepParams& P, const int scal
     const uint32_t tensor_id = h->tensor_id, slot = h->slot;
     const float s_new = ts.s_new, inv_new = ts.inv_new;
     const uint32_t seg_per_row = h->seg_per_row, div_magic = h->div_magic, n_mrows = h->n_mrows;
-    const uint64_t mrow0 = h->mrow0, index_base = h->index_base;
-    float* const ep = h->e;
+    const uint64_t mrow0 = h->mrow0;
+    // Per-lane bases, formed once per unit; the slots of a lane then differ by compile-time constants only
+    // (row step * 128 elements: a multiple of 4, so the shifts below commute with adding it).
+    uint8_t* const w_lane = wp + (FMT != FMT_INT4 ? i_first : (i_first >> 1));
+    float* const m_lane = mp + i_first;
+    float* const e_lane = ERR ? h->e + i_first : nullptr;
+    const uint32_t ctr_lane = static_cast<uint32_t>((i_first + h->index_base) >> 2);   // Philox counter of slot 0
     __syncwarp();
     if (lane == 0) mbar_arrive(empty_bar);          // the stage may be refilled
 
@@ -393,15 +398,15 @@ __device__ __forceinline__ bool consume_unit(const StepParams& P, const int scal
 #pragma unroll
     for (int k = 0; k < NS; ++k) {
         if (!FULL && r + k * kRowStep >= nrows) continue;
-        const uint64_t i0 = i_first + k * (kRowStep * 128);
+        constexpr int kSlotElems = kRowStep * 128;                   // elements between two slots of a lane
         uint32_t word[4] = {0u, 0u, 0u, 0u};
         if (RND == RND_SR) {
-            const uint4 rw = philox4x32_10(static_cast<uint32_t>((i0 + index_base) >> 2), tensor_id, P.step_lo, P.step_hi, P);
+            const uint4 rw = philox4x32_10(ctr_lane + static_cast<uint32_t>(k * (kSlotElems / 4)), tensor_id, P.step_lo, P.step_hi, P);
             word[0] = rw.x; word[1] = rw.y; word[2] = rw.z; word[3] = rw.w;
         }
         float mh[4], e_prev[4] = {0.0f, 0.0f, 0.0f, 0.0f}, e_out[4];
         if (ERR && P.inject == 2) {
-            const float4 er = *reinterpret_cast<const float4*>(ep + i0);
+            const float4 er = *reinterpret_cast<const float4*>(e_lane + k * kSlotElems);
             e_prev[0] = er.x; e_prev[1] = er.y; e_prev[2] = er.z; e_prev[3] = er.w;
         }
         // power-of-two scales make q s exact; INT4 kernels ask the step parameters (bf16 scales do too); the 8-bit
@@ -409,15 +414,15 @@ __device__ __forceinline__ bool consume_unit(const StepParams& P, const int scal
         constexpr int kExact = MODE == MODE_BLOCK32 ? 1 : (FMT == FMT_INT4 ? -1 : 0);
         const uint32_t codes = back4<FMT, OPT, RND, ERR, kExact>(P, word, s_k[k], inv_k[k], L[k], mh, e_prev, e_out);
         if (HINT) {
-            if (FMT != FMT_INT4) store_u32_first(wp + i0, codes, store_policy);
-            else store_u16_first(wp + (i0 >> 1), codes, store_policy);
-            store_f4_first(mp + i0, mh[0], mh[1], mh[2], mh[3], store_policy);
-            if (ERR) store_f4_first(ep + i0, e_out[0], e_out[1], e_out[2], e_out[3], store_policy);
+            if (FMT != FMT_INT4) store_u32_first(w_lane + k * kSlotElems, codes, store_policy);
+            else store_u16_first(w_lane + k * (kSlotElems / 2), codes, store_policy);
+            store_f4_first(m_lane + k * kSlotElems, mh[0], mh[1], mh[2], mh[3], store_policy);
+            if (ERR) store_f4_first(e_lane + k * kSlotElems, e_out[0], e_out[1], e_out[2], e_out[3], store_policy);
         } else {
-            if (FMT != FMT_INT4) *reinterpret_cast<uint32_t*>(wp + i0) = codes;
-            else *reinterpret_cast<uint16_t*>(wp + (i0 >> 1)) = static_cast<uint16_t>(codes);
-            *reinterpret_cast<float4*>(mp + i0) = make_float4(mh[0], mh[1], mh[2], mh[3]);
-            if (ERR) *reinterpret_cast<float4*>(ep + i0) = make_float4(e_out[0], e_out[1], e_out[2], e_out[3]);
+            if (FMT != FMT_INT4) *reinterpret_cast<uint32_t*>(w_lane + k * kSlotElems) = codes;
+            else *reinterpret_cast<uint16_t*>(w_lane + k * (kSlotElems / 2)) = static_cast<uint16_t>(codes);
+            *reinterpret_cast<float4*>(m_lane + k * kSlotElems) = make_float4(mh[0], mh[1], mh[2], mh[3]);
+            if (ERR) *reinterpret_cast<float4*>(e_lane + k * kSlotElems) = make_float4(e_out[0], e_out[1], e_out[2], e_out[3]);
         }
     }
     return true;
