@@ -216,6 +216,14 @@ StepParams derive_params(const eco_config& cfg, float lr_f, float beta1_f, float
         P.neg_lr_over_bc1 = -P.lr_over_bc1;
         P.neg_inv_bc2 = -P.inv_bc2;
         P.adam_coef = static_cast<float>((bc1 / lr) * (1.0 - 1.0 / b1));
+        // region of the fast square root / quotient as bounds on v~ and |m~| (see StepParams), 2^-20 inside
+        const double in = 1.0 + std::ldexp(1.0, -20), out = 1.0 - std::ldexp(1.0, -20);
+        P.fast_v_lo = static_cast<float>(std::ldexp(1.0, -80) / static_cast<double>(P.inv_bc2) * in);
+        P.fast_v_hi = static_cast<float>(std::ldexp(1.0, 60) / static_cast<double>(P.inv_bc2) * out);
+        P.fast_m_lo = static_cast<float>(std::ldexp(1.0, -60) / static_cast<double>(P.lr_over_bc1) * in);
+        P.fast_m_hi = static_cast<float>(std::ldexp(1.0, 60) / static_cast<double>(P.lr_over_bc1) * out);
+        for (float b : {P.fast_v_lo, P.fast_v_hi, P.fast_m_lo, P.fast_m_hi})
+            if (!std::isnormal(b)) P.fast_ok = 0;
     }
     P.seed_lo = static_cast<uint32_t>(seed);
     P.seed_hi = static_cast<uint32_t>(seed >> 32);
