@@ -317,7 +317,7 @@ def main():
     ap.add_argument("--workload", default="c5", choices=["c3f", "c3fs", "c1", "c2", "c3", "c4", "c5", "c3r", "c5t", "c4g", "c4d", "c3s", "c3rs", "c4s", "c5s", "c4mx", "c4mxs", "c4ds"])
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--min-seconds", type=float, default=2.0, help="blocks of --steps steps are repeated until this much has been timed")
-    ap.add_argument("--also", default="c3,c4,c4d", help="comma-separated workloads timed after the headline one and "
+    ap.add_argument("--also", default="c3,c4,c4d,c2,c1", help="comma-separated workloads timed after the headline one and "
                     "reported under other_workloads (device-resident timing only)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
