@@ -39,13 +39,18 @@ PROFILE_SOURCES = ("eco_stream_kernels.cu", "eco_device.cuh", "eco_index.h")
 
 
 def _kernel_sources_digest() -> str:
-    """SHA-256 over the sources the streaming kernels are built from: an ncu summary carries the digest of the
-    sources it was captured on, and its counters are not quoted once they have changed."""
+    """SHA-256 over the code (comments and white space stripped) of the sources the streaming kernels are built from:
+    an ncu summary carries the digest of the sources it was captured on, and its counters are not quoted once they
+    have changed."""
     import hashlib
+    import re
     h = hashlib.sha256()
     for name in PROFILE_SOURCES:
-        with open(os.path.join(ROOT, "paper_2601_22101_b200", "csrc", name), "rb") as f:
-            h.update(f.read())
+        with open(os.path.join(ROOT, "paper_2601_22101_b200", "csrc", name), "r") as f:
+            text = f.read()
+        # the code only: comments and layout do not change a kernel (no string literal in these files holds "//")
+        text = re.sub(r"//[^\n]*", "", text)
+        h.update(" ".join(text.split()).encode())
     return h.hexdigest()
 
 

@@ -2,8 +2,8 @@
 // engine.
 //
 // One CTA = 1 producer warp + 8 consumer warps, two (Adam) or three (momentum SGD) CTAs per SM.  The parameter
-// set is cut into units of 32 rows of 128 elements (4096 parameters); each CTA
-// owns a contiguous range of units.  For every unit the producer issues one
+// set is cut into units of 32 rows of 128 elements (4096 parameters), handed out to
+// the CTAs by a device-wide ticket counter.  For every unit the producer issues one
 // bulk asynchronous copy (cp.async.bulk, global -> shared, completion counted
 // on an mbarrier) per input stream -- codes, bf16 gradient, m and, for Adam, v
 // -- into a ring of shared-memory stages, and stages the unit's old scales and
