@@ -278,8 +278,13 @@ __device__ __forceinline__ bool consume_unit(const StepParams& P, const int scal
     float* const m_lane = mp + i_first;
     float* const e_lane = ERR ? h->e + i_first : nullptr;
     const uint32_t ctr_lane = static_cast<uint32_t>((i_first + h->index_base) >> 2);   // Philox counter of slot 0
-    __syncwarp();
-    if (lane == 0) mbar_arrive(empty_bar);          // the stage may be refilled
+    // (INT4 + momentum SGD with block scales hands the stage back after the row maxima instead: three CTAs per SM
+    // keep the copy engine busy anyway, and the compiler then fits the lane's state into its 72 registers)
+    constexpr bool kLateRelease = MODE == MODE_BLOCK && OPT == OPT_SGDM && FMT == FMT_INT4;
+    if (!kLateRelease) {
+        __syncwarp();
+        if (lane == 0) mbar_arrive(empty_bar);      // the stage may be refilled
+    }
 
     if (MODE == MODE_TENSOR_AMAX) {
         if (slot != cur_slot) {
@@ -313,6 +318,10 @@ __device__ __forceinline__ bool consume_unit(const StepParams& P, const int scal
         for (int k = 0; k < 4; ++k) {
             s_k[k] = __shfl_sync(0xFFFFFFFFu, s_mine, 8 * k);
             inv_k[k] = __shfl_sync(0xFFFFFFFFu, inv_mine, 8 * k);
+        }
+        if (kLateRelease) {
+            __syncwarp();
+            if (lane == 0) mbar_arrive(empty_bar);
         }
     } else if (MODE == MODE_BLOCK32) {
         // Four scale blocks of 32 elements per row, 8 lanes each: 16 maxima per warp.  Three butterfly stages inside
