@@ -71,10 +71,10 @@ struct StageLayout {
     static constexpr int kBarriers = 512;                        // 2 * kStages + 2 mbarriers, padded to 128; then the
                                                                  // per-row exchange: 32 maxima, 32 scales, 32 inverses
     static constexpr int kRowBars = 64;                          // two mbarriers of the per-row exchange
-    static constexpr int kPeerMax = 32;                          // per-row mode in a cluster: 2 x 4 partial row maxima from the peers
-    static constexpr int kClusterBars = 96;                      // ... and the two mbarriers the peers arrive on
-    static constexpr int kExchange = 128;
-    static_assert(2 * kStages * 8 <= kPeerMax, "the stage barriers end before the cluster exchange area");
+    static constexpr int kClusterBars = 96;                      // per-row mode in a cluster: the two mbarriers the peers arrive on
+    static constexpr int kExchange = 128;                        // the exchange arrays (in a cluster: 2 x 4 x 8 partial row maxima)
+    static_assert(2 * kStages * 8 <= kRowBars, "the stage barriers end before the exchange barriers");
+    static_assert(kExchange + 2 * 4 * kConsumerWarps * 4 <= kBarriers && kExchange + 96 * 4 <= kBarriers, "exchange arrays fit");
     static constexpr int kSmem = kBarriers + kStages * kBytes;
     static_assert(kBytes % 128 == 0, "stages stay 128-byte aligned");
 };
@@ -344,6 +344,32 @@ __device__ __forceinline__ bool consume_unit(const StepParams& P, const int scal
             s_k[k] = __shfl_sync(0xFFFFFFFFu, s_mine, (lane & 24) + 2 * k);
             inv_k[k] = __shfl_sync(0xFFFFFFFFu, inv_mine, (lane & 24) + 2 * k);
         }
+    } else if (MODE == MODE_ROW && cl.size > 1) {
+        // A matrix row longer than one unit: this unit is the slice of ONE matrix row that this CTA of the cluster
+        // holds.  Every warp reduces its segments to one partial maximum and hands it to every CTA of the cluster --
+        // lane r stores it into CTA r's slot (its own included) and arrives on CTA r's mbarrier -- then waits,
+        // bounded, on its own CTA's barrier for the 8 x size arrivals, reduces the 8 x size partials and derives the
+        // scale itself: one hop across the cluster, no meeting of the warps before or after it.  Slots and
+        // barriers alternate with the unit's parity, so a CTA that is a unit ahead cannot disturb one still reading.
+        float z = amax[0];
+#pragma unroll
+        for (int k = 1; k < NS; ++k) z = fmaxf(z, amax[k]);
+        z = warp_amax(z);
+        const uint32_t slot = cl.peer_max + ((row_parity * 4u + cl.rank) * kConsumerWarps + static_cast<uint32_t>(warp)) * 4u;
+        const uint32_t bar = cl.bars + row_parity * 8u;
+        if (static_cast<uint32_t>(lane) < cl.size) {
+            peer_store_f32(peer_addr(slot, lane), z);
+            peer_mbar_arrive(peer_addr(bar, lane));
+        }
+        if (!mbar_wait_cluster(bar, cl.phase, status, 9u)) return false;
+        const float* pm = cl.peer_max_ptr + row_parity * (4u * kConsumerWarps);
+        const float a = warp_amax(static_cast<uint32_t>(lane) < cl.size * kConsumerWarps ? pm[lane] : 0.0f);
+        float s_j, inv_j;
+        uint32_t bits_j;
+        make_scale_div<FMT>(a, scale_kind == SCALE_KIND_BF16, s_j, inv_j, bits_j);
+        if (cl.rank == 0u && warp == 0 && lane == 0) store_scale(sp, mrow0, scale_kind, s_j, bits_j);
+#pragma unroll
+        for (int k = 0; k < NS; ++k) { s_k[k] = s_j; inv_k[k] = inv_j; }
     } else if (MODE == MODE_ROW) {
         // One scale per matrix row = seg_per_row consecutive 128-element rows, which belong to several warps.
         // Every warp posts the maxima of its 4 rows in shared memory; after the first barrier warp w reduces
@@ -362,32 +388,14 @@ __device__ __forceinline__ bool consume_unit(const StepParams& P, const int scal
         if (!mbar_wait(row_bars, row_parity, status, 4u)) return false;
         for (uint32_t j = static_cast<uint32_t>(warp); j < n_mrows; j += kConsumerWarps) {
             const float x = static_cast<uint32_t>(lane) < seg_per_row ? xmax[j * seg_per_row + lane] : 0.0f;
-            float a = warp_amax(x);
-            bool owner = true;
-            if (cl.size > 1) {
-                // A matrix row longer than one unit: the CTAs of the cluster each hold a slice of it (this unit is ONE
-                // matrix row, so j == 0 and only warp 0 is here).  Lane r hands this CTA's partial maximum to CTA r --
-                // a store into its shared memory, then an arrival on its mbarrier -- and the warp waits, bounded, for
-                // the arrivals of all CTAs on its own.  Slots and barriers alternate with the unit's parity, so a
-                // CTA that is a unit ahead cannot disturb one that is still reading.
-                const uint32_t slot = cl.peer_max + (row_parity * 4u + cl.rank) * 4u;
-                const uint32_t bar = cl.bars + row_parity * 8u;
-                if (static_cast<uint32_t>(lane) < cl.size) {
-                    peer_store_f32(peer_addr(slot, lane), a);
-                    peer_mbar_arrive(peer_addr(bar, lane));
-                }
-                if (!mbar_wait_cluster(bar, cl.phase, status, 9u)) return false;
-                const float* pm = cl.peer_max_ptr + row_parity * 4u;
-                a = warp_amax(static_cast<uint32_t>(lane) < cl.size ? pm[lane] : 0.0f);
-                owner = cl.rank == 0u;
-            }
+            const float a = warp_amax(x);
             float s_j, inv_j;
             uint32_t bits_j;
             make_scale_div<FMT>(a, scale_kind == SCALE_KIND_BF16, s_j, inv_j, bits_j);
             if (lane == 0) {
                 xs[j] = s_j;
                 xinv[j] = inv_j;
-                if (owner) store_scale(sp, mrow0 + j, scale_kind, s_j, bits_j);
+                store_scale(sp, mrow0 + j, scale_kind, s_j, bits_j);
             }
         }
         __syncwarp();
@@ -478,8 +486,8 @@ eco_stream_kernel(const TensorDesc* __restrict__ descs, const uint32_t* __restri
         }
         mbar_init(row_bars, kConsumerWarps);
         mbar_init(row_bars + 8, kConsumerWarps);
-        mbar_init(smem_addr(smem + SL::kClusterBars), cluster_size());
-        mbar_init(smem_addr(smem + SL::kClusterBars + 8), cluster_size());
+        mbar_init(smem_addr(smem + SL::kClusterBars), cluster_size() * kConsumerWarps);       // one arrival per warp of the cluster
+        mbar_init(smem_addr(smem + SL::kClusterBars + 8), cluster_size() * kConsumerWarps);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
@@ -637,8 +645,10 @@ eco_stream_kernel(const TensorDesc* __restrict__ descs, const uint32_t* __restri
             // rows are dealt round-robin: this warp has rows warp, warp + 8, ... below nrows
             const int mine = static_cast<int>(nrows) > warp ? (static_cast<int>(nrows) - warp + kConsumerWarps - 1) / kConsumerWarps : 0;
             // (in a cluster: unit `it` uses exchange slot and barrier it & 1, whose phase parity is (it >> 1) & 1)
-            const ClusterInfo cl{crank, csize, smem_addr(smem + SL::kPeerMax), smem_addr(smem + SL::kClusterBars), (it >> 1) & 1u,
-                                 reinterpret_cast<const float*>(smem + SL::kPeerMax)};
+            // (the partial maxima of a cluster, 2 parities x 4 CTAs x 8 warps, lie where the single-CTA form keeps its
+            // exchange arrays: a launch is one or the other)
+            const ClusterInfo cl{crank, csize, smem_addr(smem + SL::kExchange), smem_addr(smem + SL::kClusterBars), (it >> 1) & 1u,
+                                 reinterpret_cast<const float*>(smem + SL::kExchange)};
             const TensorScales none{1.0f, 1.0f, 1.0f};
             if (mine == 4)
                 ok = consume_unit<FMT, OPT, RND, MODE, true, ERR, 4>(P, scale_kind, st, h, empty, warp, lane, scratch_amax, cur_slot,
