@@ -153,6 +153,12 @@ __device__ __forceinline__ void peer_store_f32(uint32_t addr, float v) {
 __device__ __forceinline__ void peer_mbar_arrive(uint32_t addr) {
     asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(addr) : "memory");
 }
+// One binary32 value into a peer's shared memory, counted as 4 bytes of the transaction the peer's mbarrier expects:
+// the barrier's wait then makes the value visible, no fence by the sender.
+__device__ __forceinline__ void peer_store_async_f32(uint32_t addr, float v, uint32_t bar_addr) {
+    asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.b32 [%0], %1, [%2];"
+                 ::"r"(addr), "r"(__float_as_uint(v)), "r"(bar_addr) : "memory");
+}
 // Bounded wait on an own mbarrier that peers arrive on (acquire at cluster scope).
 __device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity, uint32_t* status, uint32_t code) {
     const long long t0 = clock64();
@@ -347,20 +353,21 @@ __device__ __forceinline__ bool consume_unit(const StepParams& P, const int scal
     } else if (MODE == MODE_ROW && cl.size > 1) {
         // A matrix row longer than one unit: this unit is the slice of ONE matrix row that this CTA of the cluster
         // holds.  Every warp reduces its segments to one partial maximum and hands it to every CTA of the cluster --
-        // lane r stores it into CTA r's slot (its own included) and arrives on CTA r's mbarrier -- then waits,
-        // bounded, on its own CTA's barrier for the 8 x size arrivals, reduces the 8 x size partials and derives the
-        // scale itself: one hop across the cluster, no meeting of the warps before or after it.  Slots and
-        // barriers alternate with the unit's parity, so a CTA that is a unit ahead cannot disturb one still reading.
+        // lane r sends it into CTA r's slot (its own included) with an asynchronous store that counts 4 bytes on CTA r's
+        // mbarrier -- then waits, bounded, on its own CTA's barrier (8 arrivals of its own warps, each announcing the
+        // 4 x size bytes sent for it), reduces the 8 x size partials and derives the scale itself: one hop across the
+        // cluster, no fence, no meeting of the warps before or after it.  Slots and barriers alternate with the
+        // unit's parity, so a CTA that is a unit ahead cannot disturb one still reading (bytes that arrive before the
+        // announcement just run the barrier's transaction count negative for a while).
         float z = amax[0];
 #pragma unroll
         for (int k = 1; k < NS; ++k) z = fmaxf(z, amax[k]);
         z = warp_amax(z);
         const uint32_t slot = cl.peer_max + ((row_parity * 4u + cl.rank) * kConsumerWarps + static_cast<uint32_t>(warp)) * 4u;
         const uint32_t bar = cl.bars + row_parity * 8u;
-        if (static_cast<uint32_t>(lane) < cl.size) {
-            peer_store_f32(peer_addr(slot, lane), z);
-            peer_mbar_arrive(peer_addr(bar, lane));
-        }
+        // (this warp's arrival on its own barrier announces the 4 bytes each CTA of the cluster sends for it)
+        if (lane == 0) mbar_arrive_expect_tx(bar, cl.size * 4u);
+        if (static_cast<uint32_t>(lane) < cl.size) peer_store_async_f32(peer_addr(slot, lane), z, peer_addr(bar, lane));
         if (!mbar_wait_cluster(bar, cl.phase, status, 9u)) return false;
         const float* pm = cl.peer_max_ptr + row_parity * (4u * kConsumerWarps);
         const float a = warp_amax(static_cast<uint32_t>(lane) < cl.size * kConsumerWarps ? pm[lane] : 0.0f);
@@ -486,8 +493,8 @@ eco_stream_kernel(const TensorDesc* __restrict__ descs, const uint32_t* __restri
         }
         mbar_init(row_bars, kConsumerWarps);
         mbar_init(row_bars + 8, kConsumerWarps);
-        mbar_init(smem_addr(smem + SL::kClusterBars), cluster_size() * kConsumerWarps);       // one arrival per warp of the cluster
-        mbar_init(smem_addr(smem + SL::kClusterBars + 8), cluster_size() * kConsumerWarps);
+        mbar_init(smem_addr(smem + SL::kClusterBars), kConsumerWarps);       // one arrival per warp of this CTA, each announcing
+        mbar_init(smem_addr(smem + SL::kClusterBars + 8), kConsumerWarps);   // the bytes the cluster sends for that warp
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
