@@ -880,6 +880,13 @@ def test_c3_whole_set_in_one_cooperative_launch_equals_direct_load():
     _whole_set_stream_against_direct(wl.c3(), fused=1)
 
 
+def test_c3_row_wise_whole_set_streaming_and_clusters_equal_direct_load():
+    """C3's shapes with one scale per matrix row (the granularity of the paper's FP8 runs, Sec. 4.1): the streaming
+    launch for rows of up to 32 segments plus the cluster launch for the 6912-column matrices (two CTAs per row, the
+    partial maxima crossing the cluster by asynchronous stores), against the one-CTA-per-row kernel."""
+    _whole_set_stream_against_direct(wl.c3_rowwise())
+
+
 def test_c4_whole_set_streaming_equals_direct_load():
     _whole_set_stream_against_direct(wl.c4())
 
