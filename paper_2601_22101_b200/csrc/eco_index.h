@@ -38,6 +38,21 @@ ECO_HD void dequant_unit_position(uint64_t u, uint32_t units_per_row, uint32_t e
     c0 = static_cast<uint32_t>(u - row * units_per_row) * ept;      // < cols
 }
 
+// Index of the scale that unit u of that form reads.  gran: 0 per tensor, 1 per matrix row, 2 per block of `block`
+// elements of a row.  shift >= 0 says that every row is made of whole blocks of 2^shift elements, so the blocks of the
+// tensor are numbered like its elements divided by the block length and no division is needed.  Otherwise the row
+// comes from ONE 32-bit division: u < n_units <= 2^32 - 4 for every admitted shape.
+ECO_HD uint64_t dequant_scale_index(uint64_t u, uint32_t units_per_row, uint32_t ept, int gran, uint32_t block,
+                                    uint32_t scales_per_row, int shift) {
+    if (gran == 0) return 0;
+    if (gran == 2 && shift >= 0) return (u * ept) >> shift;
+    const uint32_t u32 = static_cast<uint32_t>(u);
+    const uint32_t row = u32 / units_per_row;
+    if (gran == 1) return row;
+    const uint32_t c0 = (u32 - row * units_per_row) * ept;           // < cols
+    return static_cast<uint64_t>(row) * scales_per_row + c0 / block;
+}
+
 // Tickets of a persistent launch over n_units work units walked as W regions: W * ceil(n_units / W).  The
 // unit tables hold at most 2^31 - 1 units, so this (and the few tickets every CTA draws past the end) fits 32 bits.
 ECO_HD uint32_t ticket_count(uint32_t n_units, uint32_t W) { return div_ceil_u32(n_units, W) * W; }

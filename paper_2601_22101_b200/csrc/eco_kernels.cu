@@ -498,55 +498,64 @@ template <int FMT, bool OUT_BF16, int EPT>
 __global__ void __launch_bounds__(kThreads)
 eco_dequantize_vec_kernel(const uint8_t* __restrict__ w, const void* __restrict__ scale, void* __restrict__ out,
                           const uint64_t n_units, const uint32_t units_per_row, const int gran, const uint32_t block,
-                          const uint32_t scales_per_row, const int scale_kind) {
+                          const uint32_t scales_per_row, const int scale_kind, const int shift) {
     static_assert(EPT == 4 || EPT == 8, "4 or 8 elements per thread");
     constexpr int Q = EPT / 4;
+    constexpr int U = 2;                     // units per thread and trip: both loads are issued before either is used
     // 64-bit unit counter and stride: n_units reaches 2^32 - 4 for the largest admitted tensor, and u + stride
     // must not wrap below it
-    for (uint64_t u = static_cast<uint64_t>(blockIdx.x) * kThreads + threadIdx.x; u < n_units;
-         u += static_cast<uint64_t>(gridDim.x) * kThreads) {
-        uint64_t row;
-        uint32_t c0;
-        dequant_unit_position(u, units_per_row, EPT, row, c0);
-        const uint64_t i0 = u * EPT;
-        uint32_t codes[Q];
-        if (FMT != FMT_INT4) {
-            if constexpr (EPT == 8) {
-                const uint2 r = __ldg(reinterpret_cast<const uint2*>(w + i0));
-                codes[0] = r.x; codes[1] = r.y;
+    const uint64_t stride = static_cast<uint64_t>(gridDim.x) * kThreads;
+    for (uint64_t u0 = static_cast<uint64_t>(blockIdx.x) * kThreads + threadIdx.x; u0 < n_units; u0 += U * stride) {
+        uint32_t codes[U][Q];
+        float s[U];
+#pragma unroll
+        for (int j = 0; j < U; ++j) {
+            const uint64_t u = u0 + j * stride;
+            if (u >= n_units) continue;
+            const uint64_t i0 = u * EPT;
+            if (FMT != FMT_INT4) {
+                if constexpr (EPT == 8) {
+                    const uint2 r = __ldg(reinterpret_cast<const uint2*>(w + i0));
+                    codes[j][0] = r.x; codes[j][1] = r.y;
+                } else {
+                    codes[j][0] = __ldg(reinterpret_cast<const uint32_t*>(w + i0));
+                }
             } else {
-                codes[0] = __ldg(reinterpret_cast<const uint32_t*>(w + i0));
+                if constexpr (EPT == 8) {
+                    const uint32_t r = __ldg(reinterpret_cast<const uint32_t*>(w + (i0 >> 1)));
+                    codes[j][0] = r & 0xFFFFu; codes[j][1] = r >> 16;
+                } else {
+                    codes[j][0] = __ldg(reinterpret_cast<const uint16_t*>(w + (i0 >> 1)));
+                }
             }
-        } else {
-            if constexpr (EPT == 8) {
-                const uint32_t r = __ldg(reinterpret_cast<const uint32_t*>(w + (i0 >> 1)));
-                codes[0] = r & 0xFFFFu; codes[1] = r >> 16;
+            s[j] = load_scale(scale, dequant_scale_index(u, units_per_row, EPT, gran, block, scales_per_row, shift), scale_kind);
+        }
+#pragma unroll
+        for (int j = 0; j < U; ++j) {
+            const uint64_t u = u0 + j * stride;
+            if (u >= n_units) continue;
+            const uint64_t i0 = u * EPT;
+            float x[EPT];
+#pragma unroll
+            for (int q = 0; q < Q; ++q) {
+                float val[4];
+                unpack4<FMT>(codes[j][q], val);
+#pragma unroll
+                for (int e = 0; e < 4; ++e) x[4 * q + e] = __fmul_rn(val[e], s[j]);
+            }
+            if (OUT_BF16) {
+                uint32_t p[EPT / 2];
+#pragma unroll
+                for (int t = 0; t < EPT / 2; ++t)
+                    p[t] = f32_to_bf16_bits_rne(x[2 * t]) | (f32_to_bf16_bits_rne(x[2 * t + 1]) << 16);
+                uint4* o = reinterpret_cast<uint4*>(static_cast<uint16_t*>(out) + i0);
+#pragma unroll
+                for (int t = 0; t < (EPT + 7) / 8; ++t) o[t] = make_uint4(p[4 * t], p[4 * t + 1], p[4 * t + 2], p[4 * t + 3]);
             } else {
-                codes[0] = __ldg(reinterpret_cast<const uint16_t*>(w + (i0 >> 1)));
+                float4* o = reinterpret_cast<float4*>(static_cast<float*>(out) + i0);
+#pragma unroll
+                for (int t = 0; t < Q; ++t) o[t] = make_float4(x[4 * t], x[4 * t + 1], x[4 * t + 2], x[4 * t + 3]);
             }
-        }
-        const uint64_t k = gran == 0 ? 0 : (gran == 1 ? row : row * scales_per_row + c0 / block);
-        const float s = load_scale(scale, k, scale_kind);
-        float x[EPT];
-#pragma unroll
-        for (int q = 0; q < Q; ++q) {
-            float val[4];
-            unpack4<FMT>(codes[q], val);
-#pragma unroll
-            for (int e = 0; e < 4; ++e) x[4 * q + e] = __fmul_rn(val[e], s);
-        }
-        if (OUT_BF16) {
-            uint32_t p[EPT / 2];
-#pragma unroll
-            for (int j = 0; j < EPT / 2; ++j)
-                p[j] = f32_to_bf16_bits_rne(x[2 * j]) | (f32_to_bf16_bits_rne(x[2 * j + 1]) << 16);
-            uint4* o = reinterpret_cast<uint4*>(static_cast<uint16_t*>(out) + i0);
-#pragma unroll
-            for (int j = 0; j < (EPT + 7) / 8; ++j) o[j] = make_uint4(p[4 * j], p[4 * j + 1], p[4 * j + 2], p[4 * j + 3]);
-        } else {
-            float4* o = reinterpret_cast<float4*>(static_cast<float*>(out) + i0);
-#pragma unroll
-            for (int j = 0; j < Q; ++j) o[j] = make_float4(x[4 * j], x[4 * j + 1], x[4 * j + 2], x[4 * j + 3]);
         }
     }
 }
@@ -561,9 +570,11 @@ cudaError_t launch_dequantize(const LaunchConfig& c, const uint8_t* w, const voi
         const uint64_t cap = static_cast<uint64_t>((c.sm_count > 0 ? c.sm_count : 148) * 16);
         const uint32_t g = static_cast<uint32_t>(std::max<uint64_t>(1, std::min(cap, (n_units + kThreads - 1) / kThreads)));
         const uint32_t spr = div_ceil_u32(cols, block);
+        // rows made of whole blocks of 128 or 32 elements: scale blocks are numbered like elements / block
+        const int shift = (gran == 2 && cols % block == 0u) ? (block == 128u ? 7 : (block == 32u ? 5 : -1)) : -1;
         ECO_DISPATCH_FMT(c.format, {
-            if (out_bf16) eco_dequantize_vec_kernel<F, true, 8><<<g, kThreads, 0, stream>>>(w, scale, out, n_units, cols / 8, gran, block, spr, c.scale_kind);
-            else eco_dequantize_vec_kernel<F, false, 4><<<g, kThreads, 0, stream>>>(w, scale, out, n_units, cols / 4, gran, block, spr, c.scale_kind);
+            if (out_bf16) eco_dequantize_vec_kernel<F, true, 8><<<g, kThreads, 0, stream>>>(w, scale, out, n_units, cols / 8, gran, block, spr, c.scale_kind, shift);
+            else eco_dequantize_vec_kernel<F, false, 4><<<g, kThreads, 0, stream>>>(w, scale, out, n_units, cols / 4, gran, block, spr, c.scale_kind, shift);
         })
         return cudaGetLastError();
     }

@@ -86,6 +86,30 @@ int main() {
         CHECK(row == 2 && c0 == wide - 8u);
     }
 
+    // ---- scale index of a unit of that form, against the definition (row * scales per row + column / block) ----
+    {
+        struct Shape { uint64_t rows; uint32_t cols, ept, block; };
+        const Shape shapes[] = {{(1ull << 30) - 1, 16u, 4u, 128u}, {3, 0xFFFFFFF0u, 8u, 128u}, {1ull << 20, 16384u - 128u, 8u, 128u},
+                                {5, 208u, 4u, 128u}, {7, 4096u, 8u, 32u}, {9, 48u, 8u, 32u}, {(1ull << 27), 96u, 4u, 32u}};
+        for (const Shape& sh : shapes) {
+            const uint32_t upr = sh.cols / sh.ept, spr = div_ceil_u32(sh.cols, sh.block);
+            const uint64_t n_units = dequant_units(sh.rows, sh.cols, sh.ept);
+            CHECK(n_units <= (1ull << 32) - 4);
+            const int shift = sh.cols % sh.block == 0u ? (sh.block == 128u ? 7 : 5) : -1;
+            const uint64_t probes[] = {0, 1, upr - 1ull, upr, n_units / 2, n_units / 3 + 5, n_units - 2, n_units - 1};
+            for (uint64_t u : probes) {
+                if (u >= n_units) continue;
+                uint64_t row;
+                uint32_t c0;
+                dequant_unit_position(u, upr, sh.ept, row, c0);
+                CHECK(dequant_scale_index(u, upr, sh.ept, 0, sh.block, spr, -1) == 0);
+                CHECK(dequant_scale_index(u, upr, sh.ept, 1, sh.block, spr, -1) == row);
+                CHECK(dequant_scale_index(u, upr, sh.ept, 2, sh.block, spr, -1) == row * spr + c0 / sh.block);
+                if (shift >= 0) CHECK(dequant_scale_index(u, upr, sh.ept, 2, sh.block, spr, shift) == row * spr + c0 / sh.block);
+            }
+        }
+    }
+
     // ---- 1x32 blocks inside ragged rows ----
     CHECK(block32_inside(200u, 1u, 2u) && !block32_inside(200u, 1u, 3u) && block32_inside(193u, 1u, 2u));
     CHECK(block32_inside(big, (1u << 25) - 1u, 3u) && !block32_inside(0xFFFFFF9Cu, (1u << 25) - 1u, 1u));
