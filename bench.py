@@ -314,6 +314,42 @@ def run_e2e(w, device: int, steps: int, max_host_gb: float):
                       f"held in pinned host memory"}
 
 
+def time_dequantize(peak_gbs: float, reps: int = 20):
+    """x^ = s * y of Sec. 3.1 (what the forward pass of quantized training reads every step): eco_dequantize on 256 Mi
+    elements, codes and outputs much larger than L2, CUDA events around `reps` calls after 3 warm-up calls."""
+    import torch
+    from paper_2601_22101_b200 import eco
+    rows, cols = 16384, 16384
+    n = rows * cols
+    out_rows = []
+    st = torch.cuda.current_stream().cuda_stream
+    for name, fmt, block, sdt, sd in (("fp8_e4m3_block128_f32_scales", eco.ECO_FORMAT_FP8_E4M3, 128, eco.ECO_SCALE_F32, torch.float32),
+                                      ("int4_group128_bf16_scales", eco.ECO_FORMAT_INT4, 128, eco.ECO_SCALE_BF16, torch.bfloat16)):
+        cfg = eco.Config(format=fmt, granularity=eco.ECO_SCALE_PER_BLOCK, block=block, scale_dtype=sdt)
+        cb = n // 2 if fmt == eco.ECO_FORMAT_INT4 else n
+        gen = torch.Generator(device="cuda").manual_seed(7)
+        w = torch.randint(0, 120, (cb,), dtype=torch.uint8, device="cuda", generator=gen)
+        s = torch.full((rows * (cols // block),), 1e-3, dtype=sd, device="cuda")
+        out = torch.empty(n, dtype=torch.bfloat16, device="cuda")
+        for _ in range(3):
+            eco.eco_dequantize(cfg, w, s, rows, cols, out, stream=st)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(reps):
+            eco.eco_dequantize(cfg, w, s, rows, cols, out, stream=st)
+        e1.record()
+        torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1) / reps
+        nbytes = cb + s.numel() * s.element_size() + 2 * n
+        gbs = nbytes / ms / 1e6
+        out_rows.append({"layout": name, "output": "bf16", "elements": n, "ms": ms, "achieved": gbs, "unit": "GB/s",
+                         "frac": gbs / peak_gbs, "bytes": nbytes})
+        del w, s, out
+    torch.cuda.empty_cache()
+    return out_rows
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -326,6 +362,7 @@ def main():
                     "reported under other_workloads (device-resident timing only)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-dequantize", action="store_true", help="skip the timing of eco_dequantize (1 GPU only)")
     ap.add_argument("--e2e-steps", type=int, default=5)
     ap.add_argument("--e2e-host-gb", type=float, default=24.0, help="pinned host memory the end-to-end leg may hold; the "
                     "leg runs on the first tensors of the set that fit and says which fraction that was")
@@ -471,6 +508,8 @@ def main():
             "roofline": roof,
             "other_workloads": others,
         }
+    if rank == 0 and world == 1 and not args.no_dequantize:
+        out["dequantize"] = time_dequantize(out["roofline"]["peak"])
     if not args.no_e2e:
         # every rank steps its own host-resident shard; the job's time is the slowest rank's
         barrier()

@@ -501,16 +501,16 @@ eco_dequantize_vec_kernel(const uint8_t* __restrict__ w, const void* __restrict_
                           const uint32_t scales_per_row, const int scale_kind, const int shift) {
     static_assert(EPT == 4 || EPT == 8, "4 or 8 elements per thread");
     constexpr int Q = EPT / 4;
-    constexpr int U = 2;                     // units per thread and trip: both loads are issued before either is used
+    constexpr int U = 4;                     // units per thread and trip: all loads are issued before any is used
     // 64-bit unit counter and stride: n_units reaches 2^32 - 4 for the largest admitted tensor, and u + stride
     // must not wrap below it
     const uint64_t stride = static_cast<uint64_t>(gridDim.x) * kThreads;
-    for (uint64_t u0 = static_cast<uint64_t>(blockIdx.x) * kThreads + threadIdx.x; u0 < n_units; u0 += U * stride) {
+    for (uint64_t u0 = static_cast<uint64_t>(blockIdx.x) * (U * kThreads) + threadIdx.x; u0 < n_units; u0 += U * stride) {
         uint32_t codes[U][Q];
         float s[U];
 #pragma unroll
         for (int j = 0; j < U; ++j) {
-            const uint64_t u = u0 + j * stride;
+            const uint64_t u = u0 + j * kThreads;            // the CTA's units of a trip are neighbours
             if (u >= n_units) continue;
             const uint64_t i0 = u * EPT;
             if (FMT != FMT_INT4) {
@@ -532,7 +532,7 @@ eco_dequantize_vec_kernel(const uint8_t* __restrict__ w, const void* __restrict_
         }
 #pragma unroll
         for (int j = 0; j < U; ++j) {
-            const uint64_t u = u0 + j * stride;
+            const uint64_t u = u0 + j * kThreads;            // the CTA's units of a trip are neighbours
             if (u >= n_units) continue;
             const uint64_t i0 = u * EPT;
             float x[EPT];
