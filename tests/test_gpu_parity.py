@@ -529,6 +529,7 @@ def test_per_row_scales_on_long_and_short_rows(fmt, sdt, opt):
 @pytest.mark.parametrize("fmt,gran,rnd,sdt,block", [(wl.FP8_E4M3, wl.PER_BLOCK, wl.SR, wl.SCALE_F32, 128),
                                                     (wl.FP8_E4M3, wl.PER_TENSOR, wl.RTN, wl.SCALE_F32, 128),
                                                     (wl.INT4, wl.PER_ROW, wl.SR, wl.SCALE_F32, 128),
+                                                    (wl.INT4, wl.PER_BLOCK, wl.SR, wl.SCALE_BF16, 128),
                                                     (wl.FP8_E4M3, wl.PER_BLOCK, wl.SR, wl.SCALE_E8M0, 32),
                                                     (wl.FP8_E5M2, wl.PER_BLOCK, wl.RTN, wl.SCALE_BF16, 32)])
 @pytest.mark.parametrize("injection", [eco.ECO_INJECT_EXACT, eco.ECO_INJECT_ECO])
